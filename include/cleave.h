@@ -1,0 +1,194 @@
+/*
+ * cleave.h -- C ABI of the Cleave hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The path: every training-step GEMM  C[M x N] = op(A)[M x K] . op(B)[K x N]  is cut into
+ * independent sub-GEMM tasks (an output block x a K-slice, shaped by the capabilities of a set of
+ * simulated edge devices), all tasks are executed by one persistent grouped-GEMM kernel, the
+ * K-split partial blocks are summed in a fixed order into C, and tasks lost to device churn are
+ * re-planned over the surviving devices and replayed.
+ *
+ * Conventions
+ *   - Plain C types only.  "host" / "device" on a pointer says where the memory lives.
+ *   - All matrices are row-major.  A and B hold bf16 (IEEE binary32 truncated to 16 bits), their
+ *     base addresses are 16-byte aligned and their leading dimensions are multiples of 8 elements.
+ *   - Every launch is asynchronous on the CUDA stream passed as `void* stream` (a cudaStream_t;
+ *     NULL = the legacy default stream).  Nothing synchronises except where stated.
+ *   - Return value: 0 on success, a negative CLEAVE_E_* code otherwise.  The library never prints,
+ *     throws or exits.  A plan may be used by one host thread at a time.
+ *   - There is no CPU fallback and no other backend: without a CUDA device the execution calls
+ *     return CLEAVE_E_CUDA.  Planning calls are host-only and work without a device.
+ */
+#ifndef CLEAVE_H_
+#define CLEAVE_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CLEAVE_API __attribute__((visibility("default")))
+#else
+#define CLEAVE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- error codes ------------------------------------------------------------------------- */
+#define CLEAVE_OK              0
+#define CLEAVE_E_INVAL        -1   /* bad argument (null pointer, zero size, value out of range)   */
+#define CLEAVE_E_UNSUPPORTED  -2   /* valid plan the kernels cannot run (alignment, slice count)   */
+#define CLEAVE_E_INFEASIBLE   -3   /* no plan satisfies the memory constraint                      */
+#define CLEAVE_E_NO_DEVICES   -4   /* empty device list, or no surviving device for a GEMM         */
+#define CLEAVE_E_RANGE        -5   /* task id >= number of tasks                                   */
+#define CLEAVE_E_CUDA         -6   /* a CUDA runtime / driver call failed                          */
+#define CLEAVE_E_TIMEOUT      -7   /* a bounded device-side wait expired; the kernel gave up       */
+#define CLEAVE_E_BOUNDS       -8   /* a device-side range check failed; the access was skipped     */
+#define CLEAVE_E_INCOMPLETE   -9   /* assembly read a block whose task never finished              */
+#define CLEAVE_E_NOMEM        -10  /* host or device allocation failed                             */
+
+/* ---- records ----------------------------------------------------------------------------- */
+
+/* Device record of Section 4.1 ("Communication cost", "Computation cost", "Cost model
+ * constraints"): memory capacity M_k [bytes], compute rate F_k [MFLOP/s], downlink / uplink
+ * bandwidth W^d_k, W^u_k [bytes/s], downlink / uplink overhead L^d_k, L^u_k [ns].
+ * Accepted ranges: mem_bytes <= 2^48, rates and bandwidths in [1, 2^40], latencies <= 2^40. */
+typedef struct {
+    uint64_t mem_bytes, flops_mflops, dl_Bps, ul_Bps, dl_lat_ns, ul_lat_ns;
+} cleave_device_t;
+
+/* One GEMM (Section 4.1, "Search space of GEMM": A_s in R^{m x n}, B_s in R^{n x q}; here
+ * M = m_s, K = n_s, N = q_s).
+ *   transA = 0: A stored [M x K], lda >= K.   transA = 1: stored [K x M], A[i,k] = X[k,i], lda >= M.
+ *   transB = 0: B stored [K x N], ldb >= N.   transB = 1: stored [N x K], B[k,j] = W[j,k], ldb >= K.
+ * Forward X.W is (0,0), data gradient dY.W^T is (0,1), weight gradient X^T.dY is (1,0).
+ * lda, ldb in elements.  M, N, K < 2^31. */
+typedef struct {
+    uint32_t M, N, K;
+    uint32_t lda, ldb;
+    uint8_t  transA, transB;
+    uint8_t  pad_[2];
+} cleave_gemm_t;
+
+/* One sub-GEMM task: P[alpha x beta] = A[m0:m1, k0:k1] . B[k0:k1, n0:n1]   (alpha = m1-m0 ...).
+ * The paper's shard (alpha_{s,p,k}, beta_{s,p,k}) with an added K-range; k0 = 0, k1 = K is the
+ * paper's case.  `part_off` is the offset, in fp32 elements, of the task's packed row-major block
+ * (leading dimension beta) in the partial arena.  `parent` = id for planned tasks; for a
+ * replacement task it is the failed task whose block it rewrites. */
+#define CLEAVE_TASK_SUPERSEDED 1u   /* failed and replaced: never executed or waited for again */
+#define CLEAVE_TASK_REISSUED   2u   /* created by cleave_reissue                                */
+typedef struct {
+    uint32_t id, gemm, dev, parent;
+    uint32_t m0, m1, n0, n1, k0, k1;
+    uint32_t kslice, flags;
+    uint64_t part_off;
+    uint64_t cost_ns;      /* max(downlink, uplink, compute) on `dev`, Eq. (communication-cost) */
+} cleave_task_t;           /* 64 bytes */
+
+/* Planner options.  Zero-initialise and call cleave_plan_opts_default. */
+typedef struct {
+    uint32_t gran_m, gran_n, gran_k;  /* block granularity in rows / columns / K (default 128)   */
+    uint32_t kslice_max;              /* deepest K-slice, 0 = never split for depth (default 4096)*/
+    uint32_t ksplit;                  /* 0 = automatic, else the forced number of K-slices        */
+    uint32_t ksplit_cap;              /* upper limit of the automatic choice (default 8)          */
+    uint32_t reissue_fanout;          /* pieces a failed task is cut into (default 4)             */
+    uint32_t b_in, b_out;             /* bytes per input / partial-output element (2, 4)          */
+} cleave_plan_opts_t;
+
+typedef struct cleave_plan_s cleave_plan_t;   /* opaque; owned by the library until cleave_destroy */
+
+/* ---- planning (host only) ---------------------------------------------------------------- */
+
+CLEAVE_API void cleave_plan_opts_default(cleave_plan_opts_t* o);
+
+/* Section 4.1: decide, for every GEMM, the block of rows and columns (and here the K-slice) each
+ * device computes, so that the slowest device's max(downlink, uplink, compute) time is small,
+ * under exact coverage of the output, the zero-task rule (a device gets a whole block or nothing)
+ * and the memory constraint.  Each GEMM is planned independently over the same device list.
+ *   g [host, n_gemms], d [host, n_dev], o [host or NULL = defaults]; *out receives the plan.
+ * Errors: E_INVAL, E_NO_DEVICES, E_INFEASIBLE, E_NOMEM. */
+CLEAVE_API int cleave_plan(const cleave_gemm_t* g, uint32_t n_gemms, const cleave_device_t* d, uint32_t n_dev,
+                const cleave_plan_opts_t* o, cleave_plan_t** out);
+
+/* Equal shares (the homogeneous case of Appendix A): rows in grid_m parts, columns in grid_n
+ * parts, K in ksplit parts; part sizes floor(x/parts), the first x mod parts one larger.  One
+ * implicit device per task (unbounded memory, 1 TFLOP/s, 1 GB/s links, no latency).
+ * o may be NULL.  Errors: E_INVAL. */
+CLEAVE_API int cleave_plan_uniform(const cleave_gemm_t* g, uint32_t n_gemms, uint32_t grid_m, uint32_t grid_n,
+                        uint32_t ksplit, const cleave_plan_opts_t* o, cleave_plan_t** out);
+
+CLEAVE_API uint32_t cleave_plan_num_tasks(const cleave_plan_t* p);        /* planned + reissued             */
+CLEAVE_API uint32_t cleave_plan_num_original(const cleave_plan_t* p);     /* planned only                   */
+CLEAVE_API const cleave_task_t* cleave_plan_tasks(const cleave_plan_t* p);/* host, id order; valid until the
+                                                                  next cleave_reissue / destroy  */
+CLEAVE_API uint64_t cleave_plan_arena_elems(const cleave_plan_t* p);      /* fp32 elements of the arena     */
+CLEAVE_API uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm);       /* S of that GEMM      */
+CLEAVE_API uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm);  /* modelled, max load  */
+CLEAVE_API uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm);     /* water-fill level    */
+CLEAVE_API uint32_t cleave_plan_num_tiles(const cleave_plan_t* p);        /* work units of the exec kernel  */
+
+/* Host-made failures (Section 3.2, "Device departures are detected via disconnect events"): the
+ * listed tasks are skipped by every later cleave_exec / cleave_reissue launch, as if their device
+ * had left before returning its block.  Replaces the previous list; n = 0 clears it.
+ * ids [host, n].  Errors: E_RANGE. */
+CLEAVE_API int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t n);
+
+/* ---- execution (device) ------------------------------------------------------------------ */
+
+/* Runs every live, non-dropped task: P_t = A[m0:m1,k0:k1] . B[k0:k1,n0:n1], bf16 inputs, fp32
+ * accumulation, written to partials + part_off (Section 4.1: each device computes
+ * A'_{s,p,k} o B'_{s,p,k}, a block of O_s).  Marks each finished task in the plan's bookkeeping.
+ *   A, B [host arrays of n_gemms device pointers]; partials [device, >= arena_elems floats,
+ *   128-byte aligned].  The first call on a plan creates its device mirrors (allocates).
+ * Requirements on the plan (else E_UNSUPPORTED): k0 a multiple of 64 and k1 a multiple of 64 or
+ * equal to K; m0 a multiple of 8 when transA = 1; n0 a multiple of 8 when transB = 0.
+ * Errors: E_INVAL, E_UNSUPPORTED, E_CUDA, E_NOMEM. */
+CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
+                void* stream);
+
+/* Parameter-server aggregation (Section 3.1 / 3.2: the server "aggregates the computed outputs";
+ * with a K-split it is a sum): C_g[i,j] = sum over the K-slices s of the partial block covering
+ * (i,j) in slice s, as a balanced pairwise tree over adjacent slices padded with +0.0 to a power
+ * of two -- a fixed order, so the result is deterministic.
+ *   partials [device]; C [host array of n_gemms device pointers], C_g fp32 row-major, ld = N.
+ * If a task that feeds C never finished, the device status becomes E_INCOMPLETE (see
+ * cleave_status); the sums are still written.  At most 32 K-slices (else E_UNSUPPORTED). */
+CLEAVE_API int cleave_assemble(cleave_plan_t* p, const float* partials, float* const* C, void* stream);
+
+/* Churn recovery (Section 4.2): the failed tasks' devices are dead for their GEMM; every failed
+ * task is cut by rows into at most reissue_fanout pieces; each piece goes to the surviving device
+ * that finishes it earliest under the cache-aware cost (rows / columns a survivor already holds
+ * cost no downlink; no downlink latency term), largest piece first; surviving assignments stay
+ * fixed.  The pieces are appended to the task list, run like cleave_exec and write into the
+ * failed tasks' blocks, so the arena layout and cleave_assemble are unchanged.
+ *   failed [host, n].  n = 0: synchronises the stream and takes every live task the bookkeeping
+ *   shows unfinished.  Errors: E_RANGE, E_INVAL (already superseded), E_NO_DEVICES, E_INFEASIBLE,
+ *   and those of cleave_exec. */
+CLEAVE_API int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t n,
+                   const void* const* A, const void* const* B, float* partials, void* stream);
+
+/* Host-only half of cleave_reissue: appends the replacement tasks for `failed` (same rules, same
+ * errors) without launching anything; *first_new receives the id of the first new task.  The new
+ * tasks run at the next cleave_exec.  Works without a CUDA device. */
+CLEAVE_API int cleave_replan(cleave_plan_t* p, const uint32_t* failed, uint32_t n, uint32_t* first_new);
+
+/* Synchronises `stream` and returns the device status: 0, E_TIMEOUT, E_BOUNDS or E_INCOMPLETE
+ * (the most severe seen since the last cleave_exec), or E_CUDA. */
+CLEAVE_API int cleave_status(cleave_plan_t* p, void* stream);
+
+/* Number of finished tiles of each task, copied to host (synchronises the stream).
+ * done [host, cleave_plan_num_tasks entries].  A task is finished when the count equals
+ * cleave_task_num_tiles. */
+CLEAVE_API int cleave_done_counts(cleave_plan_t* p, uint32_t* done, void* stream);
+CLEAVE_API uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task);
+
+/* Device time of the last exec-kernel and assembly-kernel launches on this plan, in
+ * milliseconds, measured with CUDA events on the launching stream (synchronises those events). */
+CLEAVE_API int cleave_last_kernel_ms(cleave_plan_t* p, float* exec_ms, float* assemble_ms);
+
+CLEAVE_API void cleave_destroy(cleave_plan_t* p);
+CLEAVE_API const char* cleave_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLEAVE_H_ */

@@ -1,0 +1,418 @@
+// C ABI of the library (see include/cleave.h): argument checks, the plan's device mirrors, TMA
+// tensor maps, and the launches.  All compute happens in the kernels of kernels.cu.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "cleave.h"
+#include "kernels.cuh"
+#include "plan_internal.hpp"
+
+namespace cleave {
+
+struct DeviceState {
+    int device = -1;
+    int sm_count = 0;
+    cleave_task_t* tasks = nullptr;   uint32_t tasks_cap = 0, tasks_n = 0;
+    TileDesc* tiles = nullptr;        uint32_t tiles_cap = 0, tiles_n = 0;
+    uint8_t* dropped = nullptr;
+    uint32_t* done = nullptr;
+    uint32_t* ntiles = nullptr;
+    uint32_t* failed_ids = nullptr;
+    unsigned int* words = nullptr;    // [0] ticket, [1] status, [2] failed count
+    CUtensorMap* maps = nullptr;
+    AsmItem* asm_items = nullptr;
+    AsmRef* asm_refs = nullptr;
+    float** c_ptrs = nullptr;
+    uint32_t* ldcs = nullptr;
+    std::vector<const void*> last_a, last_b;
+    std::vector<float*> last_c;
+    bool drops_dirty = true;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};   // exec begin/end, assemble begin/end
+    bool ev_exec = false, ev_asm = false;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows x cols] matrix with row stride ld: boxes of
+// 64 (contiguous) x 64 elements, 128-byte swizzle, zero fill outside the matrix.
+int encode_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return CLEAVE_E_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {kBlockK, kSubRows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
+}
+
+template <typename T>
+int dev_alloc(T** p, size_t n) {
+    if (n == 0) n = 1;
+    return cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T)) == cudaSuccess ? 0 : CLEAVE_E_NOMEM;
+}
+
+#define CU_TRY(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return CLEAVE_E_CUDA; } } while (0)
+#define RC_TRY(x) do { int rc_ = (x); if (rc_) return rc_; } while (0)
+
+// Creates the mirrors on first use and brings the growing tables (tasks, tiles) up to date.
+int sync_device_state(cleave_plan_s* p, cudaStream_t st) {
+    if (!p->dev) {
+        int ndev = 0;
+        if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return CLEAVE_E_CUDA; }
+        DeviceState* d = new (std::nothrow) DeviceState();
+        if (!d) return CLEAVE_E_NOMEM;
+        p->dev = d;
+        CU_TRY(cudaGetDevice(&d->device));
+        CU_TRY(cudaDeviceGetAttribute(&d->sm_count, cudaDevAttrMultiProcessorCount, d->device));
+        int cc_major = 0;
+        CU_TRY(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, d->device));
+        if (cc_major != 10) return CLEAVE_E_UNSUPPORTED;
+        CU_TRY(exec_kernel_prepare());
+        RC_TRY(dev_alloc(&d->words, 4));
+        CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
+        RC_TRY(dev_alloc(&d->maps, 2 * p->gemms.size()));
+        RC_TRY(dev_alloc(&d->c_ptrs, p->gemms.size()));
+        RC_TRY(dev_alloc(&d->ldcs, p->gemms.size()));
+        std::vector<uint32_t> ldc;
+        for (auto& g : p->gemms) ldc.push_back(g.N);
+        CU_TRY(cudaMemcpyAsync(d->ldcs, ldc.data(), ldc.size() * 4, cudaMemcpyHostToDevice, st));
+        RC_TRY(dev_alloc(&d->asm_items, p->asm_items.size()));
+        RC_TRY(dev_alloc(&d->asm_refs, p->asm_refs.size()));
+        CU_TRY(cudaMemcpyAsync(d->asm_items, p->asm_items.data(), p->asm_items.size() * sizeof(AsmItem), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->asm_refs, p->asm_refs.data(), p->asm_refs.size() * sizeof(AsmRef), cudaMemcpyHostToDevice, st));
+        for (auto& e : d->ev) CU_TRY(cudaEventCreate(&e));
+    }
+    DeviceState* d = p->dev;
+    const uint32_t nt = (uint32_t)p->tasks.size(), nl = (uint32_t)p->tiles.size();
+    if (nt > d->tasks_cap) {
+        // grow: the bookkeeping words of finished tasks must survive
+        const uint32_t cap = std::max(nt, d->tasks_cap * 2);
+        cleave_task_t* tasks; uint8_t* dropped; uint32_t *done, *ntiles, *failed;
+        RC_TRY(dev_alloc(&tasks, cap)); RC_TRY(dev_alloc(&dropped, cap)); RC_TRY(dev_alloc(&done, cap));
+        RC_TRY(dev_alloc(&ntiles, cap)); RC_TRY(dev_alloc(&failed, cap));
+        CU_TRY(cudaMemsetAsync(done, 0, cap * 4, st));
+        if (d->tasks_n) CU_TRY(cudaMemcpyAsync(done, d->done, d->tasks_n * 4, cudaMemcpyDeviceToDevice, st));
+        CU_TRY(cudaStreamSynchronize(st));
+        cudaFree(d->tasks); cudaFree(d->dropped); cudaFree(d->done); cudaFree(d->ntiles); cudaFree(d->failed_ids);
+        d->tasks = tasks; d->dropped = dropped; d->done = done; d->ntiles = ntiles; d->failed_ids = failed;
+        d->tasks_cap = cap;
+        d->drops_dirty = true;
+    }
+    // task records are re-sent in full: reissue changes the flags of old tasks as well
+    if (nt != d->tasks_n || d->drops_dirty) {
+        CU_TRY(cudaMemcpyAsync(d->tasks, p->tasks.data(), nt * sizeof(cleave_task_t), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->ntiles, p->task_ntiles.data(), nt * 4, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->dropped, p->dropped.data(), nt, cudaMemcpyHostToDevice, st));
+        d->tasks_n = nt;
+        d->drops_dirty = false;
+    }
+    if (nl > d->tiles_cap) {
+        const uint32_t cap = std::max(nl, d->tiles_cap * 2);
+        TileDesc* tiles;
+        RC_TRY(dev_alloc(&tiles, cap));
+        if (d->tiles_n) CU_TRY(cudaMemcpyAsync(tiles, d->tiles, d->tiles_n * sizeof(TileDesc), cudaMemcpyDeviceToDevice, st));
+        CU_TRY(cudaStreamSynchronize(st));
+        cudaFree(d->tiles);
+        d->tiles = tiles; d->tiles_cap = cap;
+    }
+    if (nl > d->tiles_n) {
+        CU_TRY(cudaMemcpyAsync(d->tiles + d->tiles_n, p->tiles.data() + d->tiles_n, (nl - d->tiles_n) * sizeof(TileDesc),
+                               cudaMemcpyHostToDevice, st));
+        d->tiles_n = nl;
+    }
+    return 0;
+}
+
+int update_maps(cleave_plan_s* p, const void* const* A, const void* const* B, cudaStream_t st) {
+    DeviceState* d = p->dev;
+    const size_t n = p->gemms.size();
+    bool same = d->last_a.size() == n;
+    for (size_t i = 0; same && i < n; ++i) same = (d->last_a[i] == A[i] && d->last_b[i] == B[i]);
+    if (same) return 0;
+    std::vector<CUtensorMap> host(2 * n);
+    for (size_t i = 0; i < n; ++i) {
+        const cleave_gemm_t& g = p->gemms[i];
+        if (!A[i] || !B[i] || ((uintptr_t)A[i] & 15) || ((uintptr_t)B[i] & 15)) return CLEAVE_E_INVAL;
+        // stored shapes: A is [M x K] or, transposed, [K x M]; B is [K x N] or, transposed, [N x K]
+        RC_TRY(g.transA ? encode_map(&host[2 * i], A[i], g.K, g.M, g.lda) : encode_map(&host[2 * i], A[i], g.M, g.K, g.lda));
+        RC_TRY(g.transB ? encode_map(&host[2 * i + 1], B[i], g.N, g.K, g.ldb) : encode_map(&host[2 * i + 1], B[i], g.K, g.N, g.ldb));
+    }
+    // pageable source: the copy is staged before the call returns, so `host` may go out of scope
+    CU_TRY(cudaMemcpyAsync(d->maps, host.data(), host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, st));
+    d->last_a.assign(A, A + n);
+    d->last_b.assign(B, B + n);
+    return 0;
+}
+
+int check_exec_args(cleave_plan_s* p, const void* const* A, const void* const* B, float* partials) {
+    if (!p || !A || !B || !partials) return CLEAVE_E_INVAL;
+    if ((uintptr_t)partials & 127) return CLEAVE_E_INVAL;
+    if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
+    for (const auto& g : p->gemms) {
+        const uint32_t need_a = g.transA ? g.M : g.K, need_b = g.transB ? g.K : g.N;
+        if (g.lda < need_a || g.ldb < need_b) return CLEAVE_E_INVAL;
+    }
+    return 0;
+}
+
+int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, uint32_t task_begin, uint32_t task_end,
+              int clear_status, float* partials, cudaStream_t st) {
+    DeviceState* d = p->dev;
+    CU_TRY(launch_arm_queue(d->tiles, tile_begin, tile_end, d->tasks, d->dropped, d->done, task_begin, task_end,
+                            d->words + 0, d->words + 1, clear_status, st));
+    if (tile_end > tile_begin) {
+        const uint32_t grid = std::min<uint32_t>((uint32_t)d->sm_count, tile_end - tile_begin);
+        CU_TRY(cudaEventRecord(d->ev[0], st));
+        CU_TRY(launch_exec(grid, d->tiles, tile_end, d->words + 0, d->maps, partials, d->done, d->words + 1, st));
+        CU_TRY(cudaEventRecord(d->ev[1], st));
+        d->ev_exec = true;
+    }
+    return 0;
+}
+
+int status_to_code(unsigned int s) {
+    if (s & STATUS_TIMEOUT) return CLEAVE_E_TIMEOUT;
+    if (s & STATUS_BOUNDS) return CLEAVE_E_BOUNDS;
+    if (s & STATUS_INCOMPLETE) return CLEAVE_E_INCOMPLETE;
+    return 0;
+}
+
+}  // namespace
+
+void device_state_free(DeviceState* d) {
+    if (!d) return;
+    cudaFree(d->tasks); cudaFree(d->tiles); cudaFree(d->dropped); cudaFree(d->done); cudaFree(d->ntiles);
+    cudaFree(d->failed_ids); cudaFree(d->words); cudaFree(d->maps); cudaFree(d->asm_items); cudaFree(d->asm_refs);
+    cudaFree(d->c_ptrs); cudaFree(d->ldcs);
+    for (auto& e : d->ev) if (e) cudaEventDestroy(e);
+    cudaGetLastError();
+    delete d;
+}
+
+}  // namespace cleave
+
+using namespace cleave;
+
+extern "C" {
+
+void cleave_plan_opts_default(cleave_plan_opts_t* o) {
+    if (!o) return;
+    o->gran_m = o->gran_n = o->gran_k = 128;
+    o->kslice_max = 4096;
+    o->ksplit = 0;
+    o->ksplit_cap = 8;
+    o->reissue_fanout = 4;
+    o->b_in = 2;
+    o->b_out = 4;
+}
+
+static int new_plan(const cleave_gemm_t* g, uint32_t n_gemms, const cleave_plan_opts_t* o, cleave_plan_s** out) {
+    if (!g || !n_gemms || !out) return CLEAVE_E_INVAL;
+    *out = nullptr;
+    cleave_plan_s* p = new (std::nothrow) cleave_plan_s();
+    if (!p) return CLEAVE_E_NOMEM;
+    p->gemms.assign(g, g + n_gemms);
+    if (o) p->opts = *o; else cleave_plan_opts_default(&p->opts);
+    *out = p;
+    return 0;
+}
+
+int cleave_plan(const cleave_gemm_t* g, uint32_t n_gemms, const cleave_device_t* d, uint32_t n_dev,
+                const cleave_plan_opts_t* o, cleave_plan_t** out) {
+    cleave_plan_s* p = nullptr;
+    int rc = new_plan(g, n_gemms, o, &p);
+    if (rc) return rc;
+    try {
+        if (d && n_dev) p->devices.assign(d, d + n_dev);
+        rc = plan_build(*p);
+    } catch (const std::bad_alloc&) { rc = CLEAVE_E_NOMEM; }
+    if (rc) { delete p; return rc; }
+    *out = p;
+    return 0;
+}
+
+int cleave_plan_uniform(const cleave_gemm_t* g, uint32_t n_gemms, uint32_t grid_m, uint32_t grid_n, uint32_t ksplit,
+                        const cleave_plan_opts_t* o, cleave_plan_t** out) {
+    cleave_plan_s* p = nullptr;
+    int rc = new_plan(g, n_gemms, o, &p);
+    if (rc) return rc;
+    try { rc = plan_build_uniform(*p, grid_m, grid_n, ksplit); } catch (const std::bad_alloc&) { rc = CLEAVE_E_NOMEM; }
+    if (rc) { delete p; return rc; }
+    *out = p;
+    return 0;
+}
+
+uint32_t cleave_plan_num_tasks(const cleave_plan_t* p) { return p ? (uint32_t)p->tasks.size() : 0; }
+uint32_t cleave_plan_num_original(const cleave_plan_t* p) { return p ? p->n_original : 0; }
+const cleave_task_t* cleave_plan_tasks(const cleave_plan_t* p) { return p ? p->tasks.data() : nullptr; }
+uint64_t cleave_plan_arena_elems(const cleave_plan_t* p) { return p ? p->arena_elems : 0; }
+uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->ksplit.size()) ? p->ksplit[gemm] : 0; }
+uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->makespan.size()) ? p->makespan[gemm] : 0; }
+uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->tstar.size()) ? p->tstar[gemm] : 0; }
+uint32_t cleave_plan_num_tiles(const cleave_plan_t* p) { return p ? (uint32_t)p->tiles.size() : 0; }
+uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task) { return (p && task < p->task_ntiles.size()) ? p->task_ntiles[task] : 0; }
+
+int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t n) {
+    if (!p || (n && !ids)) return CLEAVE_E_INVAL;
+    for (uint32_t i = 0; i < n; ++i) if (ids[i] >= p->tasks.size()) return CLEAVE_E_RANGE;
+    std::fill(p->dropped.begin(), p->dropped.end(), 0);
+    for (uint32_t i = 0; i < n; ++i) p->dropped[ids[i]] = 1;
+    if (p->dev) p->dev->drops_dirty = true;
+    return 0;
+}
+
+int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials, void* stream) {
+    int rc = check_exec_args(p, A, B, partials);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    try {
+        RC_TRY(sync_device_state(p, st));
+        RC_TRY(update_maps(p, A, B, st));
+    } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    return run_tiles(p, 0, (uint32_t)p->tiles.size(), 0, (uint32_t)p->tasks.size(), 1, partials, st);
+}
+
+int cleave_assemble(cleave_plan_t* p, const float* partials, float* const* C, void* stream) {
+    if (!p || !partials || !C) return CLEAVE_E_INVAL;
+    for (uint32_t s : p->ksplit) if (s > 32) return CLEAVE_E_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    DeviceState* d = p->dev;
+    const size_t n = p->gemms.size();
+    for (size_t i = 0; i < n; ++i) if (!C[i] || ((uintptr_t)C[i] & 15)) return CLEAVE_E_INVAL;
+    if (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin())) {
+        d->last_c.assign(C, C + n);
+        CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(float*), cudaMemcpyHostToDevice, st));
+    }
+    CU_TRY(launch_check_done(d->tasks, d->done, d->ntiles, d->tasks_n, d->words + 1, st));
+    CU_TRY(cudaEventRecord(d->ev[2], st));
+    for (const auto& grp : p->asm_groups)
+        CU_TRY(launch_assemble(d->asm_items, d->asm_refs, grp.item0, grp.n_items, grp.sp, partials, d->c_ptrs, d->ldcs, st));
+    CU_TRY(cudaEventRecord(d->ev[3], st));
+    d->ev_asm = true;
+    return 0;
+}
+
+int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t n, const void* const* A, const void* const* B,
+                   float* partials, void* stream) {
+    int rc = check_exec_args(p, A, B, partials);
+    if (rc) return rc;
+    if (n && !failed) return CLEAVE_E_INVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    try {
+        RC_TRY(sync_device_state(p, st));
+        std::vector<uint32_t> ids;
+        if (n == 0) {
+            // bookkeeping decides: every live task with unfinished tiles
+            DeviceState* d = p->dev;
+            CU_TRY(cudaMemsetAsync(d->words + 2, 0, sizeof(unsigned int), st));
+            CU_TRY(launch_collect_failed(d->tasks, d->done, d->ntiles, d->tasks_n, d->failed_ids, d->words + 2, st));
+            unsigned int cnt = 0;
+            CU_TRY(cudaMemcpyAsync(&cnt, d->words + 2, sizeof cnt, cudaMemcpyDeviceToHost, st));
+            CU_TRY(cudaStreamSynchronize(st));
+            ids.resize(cnt);
+            if (cnt) CU_TRY(cudaMemcpy(ids.data(), d->failed_ids, cnt * 4, cudaMemcpyDeviceToHost));
+            failed = ids.data();
+            n = cnt;
+            if (n == 0) return 0;
+        }
+        const uint32_t tiles_before = (uint32_t)p->tiles.size();
+        uint32_t first_new = 0;
+        RC_TRY(plan_reissue(*p, failed, n, &first_new));
+        if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
+        RC_TRY(sync_device_state(p, st));
+        RC_TRY(update_maps(p, A, B, st));
+        return run_tiles(p, tiles_before, (uint32_t)p->tiles.size(), first_new, (uint32_t)p->tasks.size(), 0, partials, st);
+    } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+}
+
+int cleave_replan(cleave_plan_t* p, const uint32_t* failed, uint32_t n, uint32_t* first_new) {
+    if (!p || (n && !failed) || !first_new) return CLEAVE_E_INVAL;
+    try { return plan_reissue(*p, failed, n, first_new); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+}
+
+int cleave_status(cleave_plan_t* p, void* stream) {
+    if (!p) return CLEAVE_E_INVAL;
+    if (!p->dev) return 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned int s = 0;
+    CU_TRY(cudaMemcpyAsync(&s, p->dev->words + 1, sizeof s, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    return status_to_code(s);
+}
+
+int cleave_done_counts(cleave_plan_t* p, uint32_t* done, void* stream) {
+    if (!p || !done) return CLEAVE_E_INVAL;
+    const size_t n = p->tasks.size();
+    if (!p->dev) { std::fill(done, done + n, 0u); return 0; }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t have = std::min<size_t>(n, p->dev->tasks_n);
+    std::fill(done, done + n, 0u);
+    CU_TRY(cudaMemcpyAsync(done, p->dev->done, have * 4, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    for (size_t i = 0; i < have; ++i) done[i] /= kEpiWarps;     // the kernel counts once per epilogue warp
+    return 0;
+}
+
+int cleave_last_kernel_ms(cleave_plan_t* p, float* exec_ms, float* assemble_ms) {
+    if (!p || !p->dev) return CLEAVE_E_INVAL;
+    DeviceState* d = p->dev;
+    if (exec_ms) {
+        *exec_ms = 0.f;
+        if (d->ev_exec) { CU_TRY(cudaEventSynchronize(d->ev[1])); CU_TRY(cudaEventElapsedTime(exec_ms, d->ev[0], d->ev[1])); }
+    }
+    if (assemble_ms) {
+        *assemble_ms = 0.f;
+        if (d->ev_asm) { CU_TRY(cudaEventSynchronize(d->ev[3])); CU_TRY(cudaEventElapsedTime(assemble_ms, d->ev[2], d->ev[3])); }
+    }
+    return 0;
+}
+
+void cleave_destroy(cleave_plan_t* p) {
+    if (!p) return;
+    device_state_free(p->dev);
+    delete p;
+}
+
+const char* cleave_strerror(int code) {
+    switch (code) {
+        case CLEAVE_OK: return "ok";
+        case CLEAVE_E_INVAL: return "invalid argument";
+        case CLEAVE_E_UNSUPPORTED: return "plan not supported by the kernels (alignment or slice count)";
+        case CLEAVE_E_INFEASIBLE: return "no plan satisfies the memory constraint";
+        case CLEAVE_E_NO_DEVICES: return "no (surviving) devices";
+        case CLEAVE_E_RANGE: return "task id out of range";
+        case CLEAVE_E_CUDA: return "CUDA call failed or no CUDA device";
+        case CLEAVE_E_TIMEOUT: return "device-side wait expired";
+        case CLEAVE_E_BOUNDS: return "device-side range check failed";
+        case CLEAVE_E_INCOMPLETE: return "a task feeding the assembly never finished";
+        case CLEAVE_E_NOMEM: return "out of memory";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

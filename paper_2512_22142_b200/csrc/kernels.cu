@@ -1,0 +1,558 @@
+// CUDA kernels of the Cleave hot path for sm_100a.
+//
+//   arm_queue_kernel    marks each work-list tile runnable or skipped (dropped / superseded task),
+//                       clears the bookkeeping of the tasks about to run, resets the ticket
+//   exec_kernel         persistent grouped GEMM: one CTA per SM walks the tile list through a
+//                       device-side ticket; TMA loads of 64x64 bf16 boxes into 128-byte-swizzled
+//                       shared memory, tcgen05 MMA (128 x N x 16, bf16 -> fp32) accumulating in
+//                       tensor memory, epilogue warps copy the accumulator to the task's packed
+//                       partial block and count the tile in the task's bookkeeping word
+//   check_done_kernel   flags E_INCOMPLETE if a live task has unfinished tiles
+//   assemble_kernel     fixed-order sum of the K-slices' partial blocks into C
+//   collect_failed_kernel  lists the live tasks whose bookkeeping shows unfinished tiles
+//
+// Every device-side wait is bounded: when a wait expires the CTA records E_TIMEOUT in the status
+// word, all its roles leave their loops, outstanding TMA copies and MMAs are drained (again with a
+// bound), tensor memory is released and the kernel returns.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels.cuh"
+
+namespace cleave {
+
+// -------------------------------------------------------------------------------------------------
+// PTX wrappers
+// -------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            unsigned int* status) {
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicOr(status, STATUS_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint32_t bar, int32_t c0, int32_t c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tensormap_acquire(const void* tmap) {
+    asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tmap) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the mbarrier once all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives lane (base + i).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of tcgen05.mma for a 128-byte-swizzled operand tile.
+//   bits  0-13 start address >> 4        bits 16-29 leading-dimension byte offset >> 4
+//   bits 32-45 stride-dimension byte offset >> 4      bits 46-47 descriptor version (1 on sm_100)
+//   bits 61-63 swizzle mode (2 = 128 bytes)
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor of tcgen05.mma.kind::f16: fp32 accumulator (bits 4-5 = 1), bf16 A and B
+// (bits 7-9 = 1, 10-12 = 1), operand major-ness (bit 15 A, bit 16 B; 1 = M/N contiguous),
+// N >> 3 in bits 17-22, M >> 4 in bits 24-28.
+__device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t m, uint32_t n, uint32_t a_mn_major, uint32_t b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major << 15) | (b_mn_major << 16) | ((n >> 3) << 17) |
+           ((m >> 4) << 24);
+}
+
+// -------------------------------------------------------------------------------------------------
+// arm_queue_kernel
+// -------------------------------------------------------------------------------------------------
+__global__ void arm_queue_kernel(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
+                                 const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
+                                 unsigned int* ticket, unsigned int* status, int clear_status) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) {
+        *ticket = tile_begin;
+        if (clear_status) *status = 0;
+    }
+    const uint32_t t = tile_begin + i;
+    if (t < tile_end) {
+        const uint32_t task = tiles[t].task;
+        const bool skip = dropped[task] || (tasks[task].flags & CLEAVE_TASK_SUPERSEDED);
+        const uint32_t f = tiles[t].flags & ~(uint32_t)TILE_VALID;
+        tiles[t].flags = skip ? f : (f | TILE_VALID);
+    }
+    const uint32_t k = task_begin + i;
+    if (k < task_end) done[k] = 0;
+}
+
+// -------------------------------------------------------------------------------------------------
+// exec_kernel
+// -------------------------------------------------------------------------------------------------
+struct __align__(16) ExecShared {
+    uint64_t full[kStages];        // TMA bytes of a stage have landed
+    uint64_t empty[kStages];       // the MMAs reading a stage have completed
+    uint64_t acc_full[kAccStages]; // an accumulator holds a finished tile
+    uint64_t acc_empty[kAccStages];// the epilogue has copied an accumulator out
+    uint64_t sched_full[kSchedSlots];
+    uint64_t sched_empty[kSchedSlots];
+    uint64_t drain;                // all MMAs completed (teardown)
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    TileDesc slot[kSchedSlots];
+};
+
+__global__ void __launch_bounds__(kExecThreads, 1)
+exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int* ticket,
+            const CUtensorMap* __restrict__ maps, float* __restrict__ partials, uint32_t* done, unsigned int* status) {
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ ExecShared sh;
+
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // operand stages, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes)
+    const uint32_t stage_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+    volatile uint32_t* abort_flag = &sh.abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh.full[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1); }
+        for (int a = 0; a < kAccStages; ++a) { mbar_init(smem_u32(&sh.acc_full[a]), 1); mbar_init(smem_u32(&sh.acc_empty[a]), kEpiWarps); }
+        for (int q = 0; q < kSchedSlots; ++q) { mbar_init(smem_u32(&sh.sched_full[q]), 1); mbar_init(smem_u32(&sh.sched_empty[q]), 2 + kEpiWarps); }
+        mbar_init(smem_u32(&sh.drain), 1);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == kMmaWarp) tmem_alloc(smem_u32(&sh.tmem_base), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp == kSchedWarp) {
+        // ---- scheduler: pulls tickets, skips dropped tiles, feeds the slot ring -----------------
+        if (lane == 0) {
+            for (uint32_t i = 0;; ++i) {
+                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+                if (!mbar_wait(smem_u32(&sh.sched_empty[q]), par ^ 1u, abort_flag, status)) break;
+                uint4 w0, w1, w2, w3;
+                bool end = false;
+                for (;;) {
+                    const uint32_t t = atomicAdd(ticket, 1u);
+                    if (t >= tile_end) { end = true; break; }
+                    const uint4* src = reinterpret_cast<const uint4*>(tiles + t);
+                    w0 = __ldg(src); w1 = __ldg(src + 1); w2 = __ldg(src + 2); w3 = __ldg(src + 3);
+                    if (w0.z & TILE_VALID) break;      // TileDesc::flags
+                }
+                uint4* dst = reinterpret_cast<uint4*>(&sh.slot[q]);
+                if (end) { w0 = make_uint4(0, 0, TILE_END, 0); w1 = w2 = w3 = make_uint4(0, 0, 0, 0); }
+                dst[0] = w0; dst[1] = w1; dst[2] = w2; dst[3] = w3;
+                mbar_arrive(smem_u32(&sh.sched_full[q]));
+                if (end) break;
+            }
+        }
+    } else if (warp == kTmaWarp) {
+        // ---- producer: TMA loads of the A and B sub-tiles of every K-block -------------------------
+        if (lane == 0) {
+            uint32_t it = 0, issued = 0, last_gemm = 0xFFFFFFFFu;
+            bool ok = true;
+            for (uint32_t i = 0; ok; ++i) {
+                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+                if (!mbar_wait(smem_u32(&sh.sched_full[q]), par, abort_flag, status)) break;
+                const TileDesc d = sh.slot[q];
+                mbar_arrive(smem_u32(&sh.sched_empty[q]));
+                if (d.flags & TILE_END) break;
+                const CUtensorMap* map_a = maps + 2 * d.gemm;
+                const CUtensorMap* map_b = map_a + 1;
+                if (d.gemm != last_gemm) { tensormap_acquire(map_a); tensormap_acquire(map_b); last_gemm = d.gemm; }
+                const bool a_mn = d.flags & TILE_A_MN, b_mn = d.flags & TILE_B_MN;   // M- / N-contiguous operand
+                const uint32_t nsub_a = d.rows > kSubRows ? 2u : 1u;
+                const uint32_t nsub_b = (d.n_mma + kSubRows - 1) / kSubRows;
+                const uint32_t tx = (nsub_a + nsub_b) * kSubBytes;
+                const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
+                for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                    const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                    if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, status)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&sh.full[s]);
+                    mbar_arrive_expect_tx(bar, tx);
+                    const uint32_t sa = stage_base + s * kStageBytes, sb = sa + kABytes;
+                    const int32_t k = (int32_t)(d.k0 + kb * kBlockK);
+                    for (uint32_t j = 0; j < nsub_a; ++j) {
+                        const int32_t m = (int32_t)(d.m_row + j * kSubRows);
+                        if (a_mn) tma_load_2d(sa + j * kSubBytes, map_a, bar, m, k);
+                        else      tma_load_2d(sa + j * kSubBytes, map_a, bar, k, m);
+                    }
+                    for (uint32_t j = 0; j < nsub_b; ++j) {
+                        const int32_t n = (int32_t)(d.n_col + j * kSubRows);
+                        if (b_mn) tma_load_2d(sb + j * kSubBytes, map_b, bar, n, k);
+                        else      tma_load_2d(sb + j * kSubBytes, map_b, bar, k, n);
+                    }
+                    ++issued;
+                }
+            }
+            // Wait for every copy still in flight before the CTA may exit (bounded).  A stage armed at
+            // iteration x completes phase (x / kStages) & 1 of its full barrier.
+            const uint32_t pending = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
+            for (uint32_t x = it - pending; x < it; ++x) {
+                const uint64_t t0 = global_timer_ns();
+                while (!mbar_try_wait(smem_u32(&sh.full[x % kStages]), (x / kStages) & 1u))
+                    if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(status, STATUS_TIMEOUT); break; }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ---- MMA issuer ----------------------------------------------------------------------------
+        if (lane == 0) {
+            uint32_t it = 0, acc_it = 0;
+            bool ok = true;
+            for (uint32_t i = 0; ok; ++i) {
+                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+                if (!mbar_wait(smem_u32(&sh.sched_full[q]), par, abort_flag, status)) break;
+                const TileDesc d = sh.slot[q];
+                mbar_arrive(smem_u32(&sh.sched_empty[q]));
+                if (d.flags & TILE_END) break;
+                const uint32_t a_mn = (d.flags & TILE_A_MN) ? 1u : 0u, b_mn = (d.flags & TILE_B_MN) ? 1u : 0u;
+                const uint32_t idesc = instr_desc_bf16(kBlockM, d.n_mma, a_mn, b_mn);
+                // K-contiguous tile: rows of 128 bytes, groups of 8 rows 1024 bytes apart; a 16-element K
+                // step is 32 bytes inside the swizzled row.  M/N-contiguous tile: 64-element groups along
+                // M/N are kSubBytes apart (leading offset), groups of 8 K-rows 1024 bytes apart; a K step
+                // of 16 is two such groups.
+                const uint32_t a_lbo = a_mn ? kSubBytes : 16u, a_step = a_mn ? 2048u : 32u;
+                const uint32_t b_lbo = b_mn ? kSubBytes : 16u, b_step = b_mn ? 2048u : 32u;
+                const uint32_t acc = acc_it % kAccStages, aph = (acc_it / kAccStages) & 1u;
+                if (!mbar_wait(smem_u32(&sh.acc_empty[acc]), aph ^ 1u, abort_flag, status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
+                for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                    const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                    if (!mbar_wait(smem_u32(&sh.full[s]), ph, abort_flag, status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = stage_base + s * kStageBytes, sb = sa + kABytes;
+#pragma unroll
+                    for (uint32_t k16 = 0; k16 < kBlockK / 16; ++k16) {
+                        const uint64_t a_desc = smem_desc_sw128(sa + k16 * a_step, a_lbo, 1024u);
+                        const uint64_t b_desc = smem_desc_sw128(sb + k16 * b_step, b_lbo, 1024u);
+                        umma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k16) != 0u);
+                    }
+                    umma_commit(smem_u32(&sh.empty[s]));       // stage reusable once these MMAs are done
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&sh.acc_full[acc]));      // accumulator complete
+                ++acc_it;
+            }
+            // drain: every MMA issued above has completed before tensor memory is released
+            umma_commit(smem_u32(&sh.drain));
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&sh.drain), 0u))
+                if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(status, STATUS_TIMEOUT); break; }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ---- epilogue: accumulator -> registers -> packed partial block ----------------------------
+        const uint32_t quad = warp & 3u;                     // the 32 TMEM lanes this warp may read
+        const uint32_t row = quad * 32u + lane;
+        uint32_t acc_it = 0;
+        for (uint32_t i = 0;; ++i) {
+            const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+            bool ok = mbar_wait(smem_u32(&sh.sched_full[q]), par, abort_flag, status);
+            if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            const uint32_t flags = sh.slot[q].flags, task = sh.slot[q].task, n_mma = sh.slot[q].n_mma;
+            const uint32_t rows = sh.slot[q].rows, cols = sh.slot[q].cols, ld = sh.slot[q].ld;
+            const uint64_t out_off = sh.slot[q].out_off;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.sched_empty[q]));
+            if (flags & TILE_END) break;
+            const uint32_t acc = acc_it % kAccStages, aph = (acc_it / kAccStages) & 1u;
+            ok = mbar_wait(smem_u32(&sh.acc_full[acc]), aph, abort_flag, status);
+            if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + acc * kAccCols + ((quad * 32u) << 16);
+            float* out_row = partials + out_off + (uint64_t)row * ld;
+            const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
+            const uint32_t nchunk = (n_mma + 31u) / 32u;
+            for (uint32_t c = 0; c < nchunk; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32(taddr + c * 32u, v);
+                tmem_ld_wait();
+                if (c + 1 == nchunk) {                       // accumulator fully read: hand it back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh.acc_empty[acc]));
+                }
+                if (row < rows) {
+                    const uint32_t c0 = c * 32u;
+                    if (vec_ok && c0 + 32u <= cols) {
+                        float4* dst = reinterpret_cast<float4*>(out_row + c0);
+#pragma unroll
+                        for (int x = 0; x < 8; ++x)
+                            __stcs(dst + x, make_float4(__uint_as_float(v[4 * x]), __uint_as_float(v[4 * x + 1]),
+                                                        __uint_as_float(v[4 * x + 2]), __uint_as_float(v[4 * x + 3])));
+                    } else {
+#pragma unroll
+                        for (int x = 0; x < 32; ++x)
+                            if (c0 + x < cols) out_row[c0 + x] = __uint_as_float(v[x]);
+                    }
+                }
+            }
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(&done[task], 1u);       // bookkeeping: kEpiWarps counts per tile
+            ++acc_it;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// -------------------------------------------------------------------------------------------------
+// bookkeeping kernels
+// -------------------------------------------------------------------------------------------------
+__global__ void check_done_kernel(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
+                                  uint32_t n_tasks, unsigned int* status) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_tasks) return;
+    if (tasks[i].flags & CLEAVE_TASK_SUPERSEDED) return;
+    if (done[i] != ntiles[i] * kEpiWarps) atomicOr(status, STATUS_INCOMPLETE);
+}
+
+__global__ void collect_failed_kernel(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
+                                      uint32_t n_tasks, uint32_t* out_ids, unsigned int* out_count) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_tasks) return;
+    if (tasks[i].flags & CLEAVE_TASK_SUPERSEDED) return;
+    if (done[i] != ntiles[i] * kEpiWarps) out_ids[atomicAdd(out_count, 1u)] = i;
+}
+
+// -------------------------------------------------------------------------------------------------
+// assemble_kernel
+// -------------------------------------------------------------------------------------------------
+// One CTA per item (whole rows of a rectangle of C whose K-slices each come from one block).
+// SP = slice count padded to a power of two.  The 32 lanes of a warp form G = min(SP, 8) groups;
+// group g owns the R = SP / G adjacent slices g*R .. g*R+R-1 and lane l of a group owns one float4
+// of the row.  Each lane sums its R slices as a balanced tree in registers, then a butterfly of
+// shfl_xor over the group index finishes the balanced tree over all SP slices: the order is fixed,
+// so the sum is deterministic.  Missing slices (s >= nslices) contribute +0.0f.
+template <int SP>
+__global__ void __launch_bounds__(256)
+assemble_vec_kernel(const AsmItem* __restrict__ items, const AsmRef* __restrict__ refs, uint32_t item0,
+                    const float* __restrict__ partials, float* const* __restrict__ Cptr, const uint32_t* __restrict__ ldcs) {
+    constexpr int G = SP < 8 ? SP : 8;
+    constexpr int R = SP / G;
+    constexpr int LG = 32 / G;
+    constexpr int U = 4;
+    const AsmItem it = items[item0 + blockIdx.x];
+    const uint32_t ldc = ldcs[it.gemm];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t g = lane / LG, l = lane % LG;
+    const uint32_t c4 = it.ncols >> 2;
+    const uint32_t units = it.nrows * c4;
+
+    const float* src[R];
+    uint32_t ld[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const uint32_t s = g * R + r;
+        if (s < it.nslices) { const AsmRef rf = refs[it.ref0 + s]; src[r] = partials + rf.off; ld[r] = rf.ld; }
+        else { src[r] = nullptr; ld[r] = 0; }
+    }
+    float* crow = Cptr[it.gemm] + (uint64_t)it.i0 * ldc + it.j0;
+
+    for (uint32_t base = warp * (LG * U); base < units; base += nwarps * (LG * U)) {
+        float4 acc[U];
+        uint32_t urow[U], ucol[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t unit = base + u * LG + l;
+            const bool live = unit < units;
+            urow[u] = live ? unit / c4 : 0u;
+            ucol[u] = live ? (unit - urow[u] * c4) * 4u : 0u;
+            float4 v[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                v[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (live && src[r]) v[r] = __ldcs(reinterpret_cast<const float4*>(src[r] + (uint64_t)urow[u] * ld[r] + ucol[u]));
+            }
+#pragma unroll
+            for (int w = 1; w < R; w *= 2)
+#pragma unroll
+                for (int r = 0; r < R; r += 2 * w) {
+                    v[r].x += v[r + w].x; v[r].y += v[r + w].y; v[r].z += v[r + w].z; v[r].w += v[r + w].w;
+                }
+            acc[u] = v[0];
+        }
+#pragma unroll
+        for (int off = LG; off < 32; off *= 2)
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                acc[u].x += __shfl_xor_sync(0xFFFFFFFFu, acc[u].x, off);
+                acc[u].y += __shfl_xor_sync(0xFFFFFFFFu, acc[u].y, off);
+                acc[u].z += __shfl_xor_sync(0xFFFFFFFFu, acc[u].z, off);
+                acc[u].w += __shfl_xor_sync(0xFFFFFFFFu, acc[u].w, off);
+            }
+        if (g == 0) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (base + u * LG + l < units)
+                    __stcs(reinterpret_cast<float4*>(crow + (uint64_t)urow[u] * ldc + ucol[u]), acc[u]);
+        }
+    }
+}
+
+// Any alignment, any slice count up to 32: one thread per output element, the same balanced tree.
+__global__ void assemble_scalar_kernel(const AsmItem* __restrict__ items, const AsmRef* __restrict__ refs, uint32_t item0,
+                                       const float* __restrict__ partials, float* const* __restrict__ Cptr,
+                                       const uint32_t* __restrict__ ldcs) {
+    const AsmItem it = items[item0 + blockIdx.x];
+    const uint32_t ldc = ldcs[it.gemm];
+    float* C = Cptr[it.gemm];
+    uint32_t sp = 1;
+    while (sp < it.nslices) sp *= 2;
+    const uint32_t n = it.nrows * it.ncols;
+    for (uint32_t e = threadIdx.x; e < n; e += blockDim.x) {
+        const uint32_t r = e / it.ncols, c = e - r * it.ncols;
+        float v[32];
+        for (uint32_t s = 0; s < sp; ++s) {
+            v[s] = 0.f;
+            if (s < it.nslices) { const AsmRef rf = refs[it.ref0 + s]; v[s] = partials[rf.off + (uint64_t)r * rf.ld + c]; }
+        }
+        for (uint32_t w = 1; w < sp; w *= 2)
+            for (uint32_t s = 0; s < sp; s += 2 * w) v[s] += v[s + w];
+        C[(uint64_t)(it.i0 + r) * ldc + it.j0 + c] = v[0];
+    }
+}
+
+// -------------------------------------------------------------------------------------------------
+// host-side launchers
+// -------------------------------------------------------------------------------------------------
+cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
+                             const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
+                             unsigned int* ticket, unsigned int* status, int clear_status, cudaStream_t st) {
+    uint32_t n = tile_end - tile_begin;
+    if (task_end - task_begin > n) n = task_end - task_begin;
+    if (n == 0) n = 1;
+    arm_queue_kernel<<<(n + 255) / 256, 256, 0, st>>>(tiles, tile_begin, tile_end, tasks, dropped, done, task_begin,
+                                                       task_end, ticket, status, clear_status);
+    return cudaGetLastError();
+}
+
+cudaError_t exec_kernel_prepare() {
+    return cudaFuncSetAttribute(exec_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kExecDynSmem);
+}
+
+cudaError_t launch_exec(uint32_t grid, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
+                        const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status,
+                        cudaStream_t st) {
+    exec_kernel<<<grid, kExecThreads, kExecDynSmem, st>>>(tiles, tile_end, ticket, maps, partials, done, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles, uint32_t n_tasks,
+                              unsigned int* status, cudaStream_t st) {
+    if (!n_tasks) return cudaSuccess;
+    check_done_kernel<<<(n_tasks + 255) / 256, 256, 0, st>>>(tasks, done, ntiles, n_tasks, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
+                                  uint32_t n_tasks, uint32_t* out_ids, unsigned int* out_count, cudaStream_t st) {
+    if (!n_tasks) return cudaSuccess;
+    collect_failed_kernel<<<(n_tasks + 255) / 256, 256, 0, st>>>(tasks, done, ntiles, n_tasks, out_ids, out_count);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
+                            const float* partials, float* const* Cptr, const uint32_t* ldcs, cudaStream_t st) {
+    if (!n_items) return cudaSuccess;
+    switch (sp) {
+        case 0:  assemble_scalar_kernel<<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 1:  assemble_vec_kernel<1><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 2:  assemble_vec_kernel<2><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 4:  assemble_vec_kernel<4><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 8:  assemble_vec_kernel<8><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 16: assemble_vec_kernel<16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 32: assemble_vec_kernel<32><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace cleave

@@ -1,0 +1,50 @@
+// Shared constants and launcher declarations of the CUDA kernels (internal).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "plan_internal.hpp"
+
+namespace cleave {
+
+// exec kernel geometry
+constexpr uint32_t kBlockM = 128;                    // MMA M: rows of a tile
+constexpr uint32_t kBlockNMax = 256;                 // widest MMA N
+constexpr uint32_t kBlockK = 64;                     // K per pipeline stage: 64 bf16 = one 128-byte swizzle row
+constexpr uint32_t kSubRows = 64;                    // rows (or M/N elements) per TMA box
+constexpr uint32_t kSubBytes = kSubRows * kBlockK * 2;          // 8192: one 64 x 64 bf16 box
+constexpr uint32_t kABytes = 2 * kSubBytes;          // 128 rows of A
+constexpr uint32_t kBBytes = 4 * kSubBytes;          // up to 256 columns of B
+constexpr uint32_t kStageBytes = kABytes + kBBytes;  // 49152
+constexpr int kStages = 4;
+constexpr int kAccStages = 2;                        // accumulators in tensor memory (double buffer)
+constexpr uint32_t kAccCols = 256;
+constexpr uint32_t kTmemCols = 512;
+constexpr int kSchedSlots = 4;
+constexpr uint32_t kExecDynSmem = kStages * kStageBytes + 1024;
+
+constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4, kEpiWarps = 4;
+constexpr int kExecThreads = 256;
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;     // bound of every device-side wait
+
+// device status word bits
+enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BOUNDS = 2u, STATUS_INCOMPLETE = 4u };
+
+cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
+                             const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
+                             unsigned int* ticket, unsigned int* status, int clear_status, cudaStream_t st);
+cudaError_t exec_kernel_prepare();
+cudaError_t launch_exec(uint32_t grid, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
+                        const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status, cudaStream_t st);
+cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles, uint32_t n_tasks,
+                              unsigned int* status, cudaStream_t st);
+cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
+                                  uint32_t n_tasks, uint32_t* out_ids, unsigned int* out_count, cudaStream_t st);
+// sp = padded slice count of the vectorised kernel (1, 2, 4, 8, 16, 32), 0 = scalar kernel
+cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
+                            const float* partials, float* const* Cptr, const uint32_t* ldcs, cudaStream_t st);
+
+}  // namespace cleave

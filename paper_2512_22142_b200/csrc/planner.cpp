@@ -1,0 +1,589 @@
+// Host planner: GEMM -> sub-GEMM tasks under the cost model of Section 4.1, the uniform grid, and
+// the churn re-plan of Section 4.2.  Integer arithmetic only (128-bit intermediates).
+//
+// The paper solves the plan as a MILP with a commercial solver; this is a deterministic heuristic
+// for the same objective and constraints:
+//   water-fill a makespan T* at which the devices' capacities (largest area each can finish in T*
+//   under downlink, uplink, compute and memory) add up to the work; sort the devices that can take
+//   at least one granule cell (the others stay idle: zero-task rule); group them into teams of S
+//   (one member per K-slice); deal the teams to column strips in snake order; apportion strip
+//   widths and team heights in granules by largest remainder; cut every rectangle into its S
+//   K-slices; split whatever still violates the memory constraint.
+#include <algorithm>
+#include <cstring>
+#include <map>
+#include <numeric>
+
+#include "plan_internal.hpp"
+
+namespace cleave {
+namespace {
+
+typedef unsigned __int128 u128;
+const uint64_t kNs = 1000000000ull;
+const uint64_t kTmax = 1ull << 50;
+
+inline uint64_t cdiv(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+inline u128 cdiv128(u128 a, u128 b) { return (a + b - 1) / b; }
+inline uint64_t sat64(u128 x) { return x > (u128)UINT64_MAX ? UINT64_MAX : (uint64_t)x; }
+
+// ---- cost model (Section 4.1) ---------------------------------------------------------------
+uint64_t cost_dl(uint64_t a, uint64_t b, uint64_t k, const cleave_device_t& d, uint32_t bin, bool lat) {
+    u128 t = cdiv128((u128)(a + b) * k * bin * kNs, d.dl_Bps);
+    return sat64(t + (lat ? d.dl_lat_ns : 0));
+}
+uint64_t cost_ul(uint64_t a, uint64_t b, const cleave_device_t& d, uint32_t bout) {
+    return sat64(cdiv128((u128)a * b * bout * kNs, d.ul_Bps) + d.ul_lat_ns);
+}
+uint64_t cost_comp(uint64_t a, uint64_t b, uint64_t k, const cleave_device_t& d) {
+    return sat64(cdiv128((u128)2 * a * b * k * 1000, d.flops_mflops));
+}
+uint64_t cost_task(uint64_t a, uint64_t b, uint64_t k, const cleave_device_t& d, const cleave_plan_opts_t& o) {
+    return std::max(std::max(cost_dl(a, b, k, d, o.b_in, true), cost_ul(a, b, d, o.b_out)), cost_comp(a, b, k, d));
+}
+u128 mem_task(uint64_t a, uint64_t b, uint64_t k, const cleave_plan_opts_t& o) {
+    return (u128)(a + b) * k * o.b_in + (u128)a * b * o.b_out;
+}
+
+// Side of the largest square block that fits the device's memory with slices of depth kh.
+uint64_t square_side_in_memory(uint64_t mem, uint64_t kh, const cleave_plan_opts_t& o) {
+    uint64_t lo = 0, hi = 1ull << 32;
+    while (lo < hi) {
+        uint64_t mid = lo + (hi - lo + 1) / 2;
+        u128 need = (u128)2 * mid * kh * o.b_in + (u128)mid * mid * o.b_out;
+        if (need <= mem) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// Largest output area the device can complete within T for slices of depth kh.
+uint64_t capacity_at(const cleave_device_t& d, uint64_t T, uint64_t kh, uint64_t side, const cleave_plan_opts_t& o) {
+    u128 best = (u128)side * side;                                     // memory
+    u128 a_comp = (u128)T * d.flops_mflops / ((u128)2000 * kh);        // compute
+    best = std::min(best, a_comp);
+    u128 a_ul = 0;                                                     // uplink
+    if (T > d.ul_lat_ns) a_ul = (u128)(T - d.ul_lat_ns) * d.ul_Bps / ((u128)kNs * o.b_out);
+    best = std::min(best, a_ul);
+    u128 a_dl = 0;                                                     // downlink: alpha+beta affordable, squared off
+    if (T > d.dl_lat_ns) {
+        u128 s = (u128)(T - d.dl_lat_ns) * d.dl_Bps / ((u128)kNs * kh * o.b_in);
+        a_dl = (s / 2) * (s - s / 2);
+    }
+    best = std::min(best, a_dl);
+    if (best < (u128)o.gran_m * o.gran_n) return 0;                    // cannot take one cell: idle
+    return (uint64_t)best;                                             // <= side^2 <= 2^64 - 1
+}
+
+uint64_t isqrt64(uint64_t x) {
+    uint64_t r = 0, bit = 1ull << 62;
+    while (bit > x) bit >>= 2;
+    while (bit) {
+        if (x >= r + bit) { x -= r + bit; r = (r >> 1) + bit; } else r >>= 1;
+        bit >>= 2;
+    }
+    return r;
+}
+
+// total units over weights.size() parts, at least one each, the rest by largest remainder.
+std::vector<uint32_t> apportion(uint32_t total, const std::vector<u128>& w) {
+    size_t n = w.size();
+    u128 W = 0;
+    for (u128 x : w) W += x;
+    uint32_t rest = total - (uint32_t)n;
+    std::vector<uint32_t> q(n);
+    std::vector<u128> rem(n);
+    uint32_t given = 0;
+    for (size_t i = 0; i < n; ++i) {
+        u128 prod = (u128)rest * w[i];
+        q[i] = (uint32_t)(prod / W);
+        rem[i] = prod - (u128)q[i] * W;
+        given += q[i];
+    }
+    std::vector<uint32_t> idx(n);
+    std::iota(idx.begin(), idx.end(), 0u);
+    std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) { return rem[a] > rem[b]; });
+    for (uint32_t i = 0; i < rest - given; ++i) q[idx[i]] += 1;
+    for (auto& x : q) x += 1;
+    return q;
+}
+
+std::vector<uint32_t> even_parts(uint32_t total, uint32_t parts) {
+    std::vector<uint32_t> v(parts, total / parts);
+    for (uint32_t i = 0; i < total % parts; ++i) v[i] += 1;
+    return v;
+}
+
+struct Rect { uint32_t m0, m1, n0, n1, k0, k1, s, dev; };
+
+int repair_memory(const Rect& r, const cleave_device_t& d, const cleave_plan_opts_t& o, std::vector<Rect>& out) {
+    if (mem_task(r.m1 - r.m0, r.n1 - r.n0, r.k1 - r.k0, o) <= (u128)d.mem_bytes) { out.push_back(r); return 0; }
+    uint32_t rg = (uint32_t)cdiv(r.m1 - r.m0, o.gran_m), cg = (uint32_t)cdiv(r.n1 - r.n0, o.gran_n);
+    Rect a = r, b = r;
+    if (rg >= cg && rg > 1) {
+        a.m1 = b.m0 = r.m0 + ((rg + 1) / 2) * o.gran_m;
+    } else if (cg > 1) {
+        a.n1 = b.n0 = r.n0 + ((cg + 1) / 2) * o.gran_n;
+    } else {
+        return CLEAVE_E_INFEASIBLE;
+    }
+    int rc = repair_memory(a, d, o, out);
+    return rc ? rc : repair_memory(b, d, o, out);
+}
+
+int plan_one(const cleave_gemm_t& g, const std::vector<cleave_device_t>& devs, const cleave_plan_opts_t& o,
+             uint32_t* S_out, uint64_t* tstar_out, std::vector<Rect>& rects) {
+    const uint32_t D = (uint32_t)devs.size();
+    const uint32_t Mg = (uint32_t)cdiv(g.M, o.gran_m), Ng = (uint32_t)cdiv(g.N, o.gran_n), Kg = (uint32_t)cdiv(g.K, o.gran_k);
+    uint32_t S, s_limit;
+    if (o.ksplit) {
+        S = s_limit = std::max(1u, std::min(o.ksplit, Kg));
+    } else {
+        uint64_t depth = o.kslice_max ? cdiv(g.K, o.kslice_max) : 1;
+        uint64_t fan = cdiv(D, (uint64_t)Mg * Ng);
+        s_limit = std::min(o.ksplit_cap, Kg);
+        S = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(std::max(depth, fan), s_limit));
+    }
+
+    std::vector<uint64_t> side(D), cap(D);
+    uint64_t kh = 0, tstar = 0;
+    for (;;) {
+        kh = std::min<uint64_t>(g.K, (uint64_t)o.gran_k * cdiv(Kg, S));
+        for (uint32_t k = 0; k < D; ++k) side[k] = square_side_in_memory(devs[k].mem_bytes, kh, o);
+        const u128 need = (u128)S * g.M * g.N;
+        auto total = [&](uint64_t T) {
+            u128 sum = 0;
+            for (uint32_t k = 0; k < D; ++k) sum += capacity_at(devs[k], T, kh, side[k], o);
+            return sum;
+        };
+        if (total(kTmax) >= need) {
+            uint64_t lo = 0, hi = kTmax;
+            while (lo < hi) {
+                uint64_t mid = lo + (hi - lo) / 2;
+                if (total(mid) >= need) hi = mid; else lo = mid + 1;
+            }
+            tstar = lo;
+            break;
+        }
+        if (S + 1 > s_limit) return CLEAVE_E_INFEASIBLE;
+        ++S;
+    }
+    for (uint32_t k = 0; k < D; ++k) cap[k] = capacity_at(devs[k], tstar, kh, side[k], o);
+
+    std::vector<uint32_t> active;
+    for (uint32_t k = 0; k < D; ++k) if (cap[k]) active.push_back(k);
+    std::stable_sort(active.begin(), active.end(), [&](uint32_t a, uint32_t b) { return cap[a] > cap[b]; });
+    const uint32_t n_act = (uint32_t)active.size();
+    const uint32_t n_teams = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(n_act / S, (uint64_t)Mg * Ng));
+    std::vector<u128> weight(n_teams, 0);
+    auto member = [&](uint32_t team, uint32_t s) { return active[((uint64_t)team * S + s) % n_act]; };
+    for (uint32_t j = 0; j < n_teams; ++j)
+        for (uint32_t s = 0; s < S; ++s) weight[j] += cap[member(j, s)];
+
+    uint32_t c = (uint32_t)isqrt64((uint64_t)n_teams * Ng / Mg);
+    c = std::max(1u, std::min(c, std::min(n_teams, Ng)));
+    while (cdiv(n_teams, c) > Mg) ++c;
+    std::vector<std::vector<uint32_t>> strips(c);
+    for (uint32_t j = 0; j < n_teams; ++j) {
+        uint32_t r = j % (2 * c);
+        strips[r < c ? r : 2 * c - 1 - r].push_back(j);
+    }
+    std::vector<u128> strip_w(c, 0);
+    for (uint32_t i = 0; i < c; ++i) {
+        if (strips[i].empty() || strips[i].size() > Mg) return CLEAVE_E_INFEASIBLE;
+        for (uint32_t j : strips[i]) strip_w[i] += weight[j];
+    }
+    const std::vector<uint32_t> widths = apportion(Ng, strip_w);
+    const std::vector<uint32_t> kparts = even_parts(Kg, S);
+
+    uint32_t col_g = 0;
+    for (uint32_t i = 0; i < c; ++i) {
+        const uint32_t n0 = col_g * o.gran_n, n1 = (uint32_t)std::min<uint64_t>(g.N, (uint64_t)(col_g + widths[i]) * o.gran_n);
+        std::vector<u128> tw;
+        for (uint32_t j : strips[i]) tw.push_back(weight[j]);
+        const std::vector<uint32_t> heights = apportion(Mg, tw);
+        uint32_t row_g = 0;
+        for (size_t t = 0; t < strips[i].size(); ++t) {
+            const uint32_t m0 = row_g * o.gran_m, m1 = (uint32_t)std::min<uint64_t>(g.M, (uint64_t)(row_g + heights[t]) * o.gran_m);
+            uint32_t kg = 0;
+            for (uint32_t s = 0; s < S; ++s) {
+                Rect r;
+                r.m0 = m0; r.m1 = m1; r.n0 = n0; r.n1 = n1;
+                r.k0 = kg * o.gran_k;
+                r.k1 = (uint32_t)std::min<uint64_t>(g.K, (uint64_t)(kg + kparts[s]) * o.gran_k);
+                r.s = s; r.dev = member(strips[i][t], s);
+                int rc = repair_memory(r, devs[r.dev], o, rects);
+                if (rc) return rc;
+                kg += kparts[s];
+            }
+            row_g += heights[t];
+        }
+        col_g += widths[i];
+    }
+    *S_out = S;
+    *tstar_out = tstar;
+    return 0;
+}
+
+inline uint64_t round_up32(uint64_t x) { return (x + 31) / 32 * 32; }
+
+void emit_tasks(cleave_plan_s& p, uint32_t gi, const std::vector<Rect>& rects) {
+    std::map<uint32_t, u128> load;
+    for (const Rect& r : rects) {
+        cleave_task_t t;
+        std::memset(&t, 0, sizeof t);
+        t.id = t.parent = (uint32_t)p.tasks.size();
+        t.gemm = gi; t.dev = r.dev;
+        t.m0 = r.m0; t.m1 = r.m1; t.n0 = r.n0; t.n1 = r.n1; t.k0 = r.k0; t.k1 = r.k1;
+        t.kslice = r.s; t.flags = 0;
+        t.part_off = p.arena_elems;
+        t.cost_ns = cost_task(r.m1 - r.m0, r.n1 - r.n0, r.k1 - r.k0, p.devices[r.dev], p.opts);
+        p.arena_elems += round_up32((uint64_t)(r.m1 - r.m0) * (r.n1 - r.n0));
+        load[r.dev] += t.cost_ns;
+        p.tasks.push_back(t);
+    }
+    u128 worst = 0;
+    for (auto& kv : load) worst = std::max(worst, kv.second);
+    p.makespan.push_back(sat64(worst));
+    p.dead.emplace_back();
+}
+
+int validate_common(const cleave_plan_s& p) {
+    const cleave_plan_opts_t& o = p.opts;
+    if (!o.gran_m || !o.gran_n || !o.gran_k || !o.b_in || !o.b_out || !o.reissue_fanout || !o.ksplit_cap) return CLEAVE_E_INVAL;
+    if (o.b_in > 16 || o.b_out > 16) return CLEAVE_E_INVAL;
+    if (p.gemms.empty()) return CLEAVE_E_INVAL;
+    for (const auto& g : p.gemms) {
+        if (!g.M || !g.N || !g.K || g.M >= (1u << 31) || g.N >= (1u << 31) || g.K >= (1u << 31)) return CLEAVE_E_INVAL;
+        if (g.transA > 1 || g.transB > 1) return CLEAVE_E_INVAL;
+    }
+    return 0;
+}
+
+void finish(cleave_plan_s& p) {
+    p.n_original = (uint32_t)p.tasks.size();
+    p.dropped.assign(p.tasks.size(), 0);
+    p.task_ntiles.clear();
+    p.tiles.clear();
+    build_tiles(p, 0);
+    p.tiles_original = (uint32_t)p.tiles.size();
+}
+
+}  // namespace
+
+int plan_build(cleave_plan_s& p) {
+    int rc = validate_common(p);
+    if (rc) return rc;
+    if (p.devices.empty()) return CLEAVE_E_NO_DEVICES;
+    for (const auto& d : p.devices) {
+        if (d.mem_bytes > (1ull << 48) || !d.flops_mflops || d.flops_mflops > (1ull << 40) || !d.dl_Bps ||
+            d.dl_Bps > (1ull << 40) || !d.ul_Bps || d.ul_Bps > (1ull << 40) || d.dl_lat_ns > (1ull << 40) ||
+            d.ul_lat_ns > (1ull << 40))
+            return CLEAVE_E_INVAL;
+    }
+    for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
+        std::vector<Rect> rects;
+        uint32_t S = 0; uint64_t tstar = 0;
+        rc = plan_one(p.gemms[gi], p.devices, p.opts, &S, &tstar, rects);
+        if (rc) return rc;
+        p.ksplit.push_back(S);
+        p.tstar.push_back(tstar);
+        emit_tasks(p, gi, rects);
+    }
+    finish(p);
+    return build_assembly(p);
+}
+
+int plan_build_uniform(cleave_plan_s& p, uint32_t gm, uint32_t gn, uint32_t ks) {
+    int rc = validate_common(p);
+    if (rc) return rc;
+    if (!gm || !gn || !ks) return CLEAVE_E_INVAL;
+    for (const auto& g : p.gemms) if (gm > g.M || gn > g.N || ks > g.K) return CLEAVE_E_INVAL;
+    if ((u128)gm * gn * ks > (1u << 24)) return CLEAVE_E_INVAL;
+    cleave_device_t unit = {1ull << 48, 1000000ull, 1000000000ull, 1000000000ull, 0, 0};
+    p.devices.assign((size_t)gm * gn * ks, unit);
+    for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
+        const cleave_gemm_t& g = p.gemms[gi];
+        const auto hm = even_parts(g.M, gm), wn = even_parts(g.N, gn), dk = even_parts(g.K, ks);
+        std::vector<Rect> rects;
+        uint32_t m0 = 0;
+        for (uint32_t i = 0; i < gm; ++i) {
+            uint32_t n0 = 0;
+            for (uint32_t j = 0; j < gn; ++j) {
+                uint32_t k0 = 0;
+                for (uint32_t s = 0; s < ks; ++s) {
+                    Rect r = {m0, m0 + hm[i], n0, n0 + wn[j], k0, k0 + dk[s], s, (uint32_t)rects.size()};
+                    rects.push_back(r);
+                    k0 += dk[s];
+                }
+                n0 += wn[j];
+            }
+            m0 += hm[i];
+        }
+        p.ksplit.push_back(ks);
+        p.tstar.push_back(0);
+        emit_tasks(p, gi, rects);
+    }
+    finish(p);
+    return build_assembly(p);
+}
+
+// ---- churn recovery (Section 4.2) -------------------------------------------------------------
+namespace {
+// integers of [lo, hi) outside the union of the intervals
+uint32_t uncovered(uint32_t lo, uint32_t hi, std::vector<std::pair<uint32_t, uint32_t>> iv) {
+    std::sort(iv.begin(), iv.end());
+    uint32_t cur = lo, cov = 0;
+    for (auto& x : iv) {
+        uint32_t a = std::max(x.first, cur), b = std::min(x.second, hi);
+        if (b > a) { cov += b - a; cur = b; }
+    }
+    return (hi - lo) - cov;
+}
+}  // namespace
+
+int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t* first_new) {
+    const cleave_plan_opts_t& o = p.opts;
+    *first_new = (uint32_t)p.tasks.size();
+    std::vector<uint32_t> F(failed, failed + n);
+    std::sort(F.begin(), F.end());
+    F.erase(std::unique(F.begin(), F.end()), F.end());
+    for (uint32_t f : F) {
+        if (f >= p.tasks.size()) return CLEAVE_E_RANGE;
+        if (p.tasks[f].flags & CLEAVE_TASK_SUPERSEDED) return CLEAVE_E_INVAL;
+    }
+    if (F.empty()) return 0;
+    std::vector<uint8_t> is_failed(p.tasks.size(), 0);
+    for (uint32_t f : F) is_failed[f] = 1;
+
+    struct Round { std::vector<uint32_t> live; std::set<uint32_t> dead; std::map<uint32_t, u128> load;
+                   std::map<uint32_t, std::vector<uint32_t>> held; };
+    std::map<uint32_t, Round> rounds;                     // per affected GEMM
+    for (uint32_t f : F) {
+        Round& r = rounds[p.tasks[f].gemm];
+        r.dead.insert(p.tasks[f].dev);
+    }
+    for (auto& kv : rounds) {
+        Round& r = kv.second;
+        r.dead.insert(p.dead[kv.first].begin(), p.dead[kv.first].end());
+    }
+    for (const cleave_task_t& t : p.tasks) {
+        auto it = rounds.find(t.gemm);
+        if (it == rounds.end() || (t.flags & CLEAVE_TASK_SUPERSEDED) || is_failed[t.id]) continue;
+        if (it->second.dead.count(t.dev)) continue;
+        it->second.held[t.dev].push_back(t.id);
+    }
+    for (auto& kv : rounds) {
+        for (auto& h : kv.second.held) { kv.second.live.push_back(h.first); kv.second.load[h.first] = 0; }
+        if (kv.second.live.empty()) return CLEAVE_E_NO_DEVICES;
+    }
+
+    std::vector<cleave_task_t> pieces;
+    uint32_t next_id = (uint32_t)p.tasks.size();
+    for (uint32_t f : F) {
+        const cleave_task_t t = p.tasks[f];
+        const uint32_t beta = t.n1 - t.n0;
+        const uint32_t rows_g = (uint32_t)cdiv(t.m1 - t.m0, o.gran_m);
+        const uint32_t parts = std::min(o.reissue_fanout, rows_g);
+        uint32_t r0 = t.m0;
+        for (uint32_t hg : even_parts(rows_g, parts)) {
+            cleave_task_t c = t;
+            c.id = next_id++;
+            c.parent = f;
+            c.dev = UINT32_MAX;
+            c.m0 = r0;
+            c.m1 = (uint32_t)std::min<uint64_t>(t.m1, (uint64_t)r0 + (uint64_t)hg * o.gran_m);
+            c.flags = CLEAVE_TASK_REISSUED;
+            c.part_off = t.part_off + (uint64_t)(r0 - t.m0) * beta;
+            c.cost_ns = 0;
+            pieces.push_back(c);
+            r0 = c.m1;
+        }
+    }
+
+    std::vector<uint32_t> order(pieces.size());
+    std::iota(order.begin(), order.end(), 0u);
+    auto work = [&](const cleave_task_t& t) { return (u128)2 * (t.m1 - t.m0) * (t.n1 - t.n0) * (t.k1 - t.k0); };
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return work(pieces[a]) > work(pieces[b]); });
+
+    auto task_at = [&](uint32_t id) -> const cleave_task_t& {
+        return id < p.tasks.size() ? p.tasks[id] : pieces[id - p.tasks.size()];
+    };
+    for (uint32_t pi : order) {
+        cleave_task_t& pc = pieces[pi];
+        Round& r = rounds[pc.gemm];
+        const uint32_t a = pc.m1 - pc.m0, b = pc.n1 - pc.n0, kk = pc.k1 - pc.k0;
+        bool found = false;
+        u128 best_cand = 0; uint64_t best_cost = 0; uint32_t best_dev = 0;
+        for (uint32_t k : r.live) {
+            const cleave_device_t& d = p.devices[k];
+            if (mem_task(a, b, kk, o) > (u128)d.mem_bytes) continue;
+            std::vector<std::pair<uint32_t, uint32_t>> rows, cols;
+            for (uint32_t hid : r.held[k]) {
+                const cleave_task_t& h = task_at(hid);
+                if (h.k0 <= pc.k0 && h.k1 >= pc.k1) { rows.emplace_back(h.m0, h.m1); cols.emplace_back(h.n0, h.n1); }
+            }
+            const uint32_t a_hat = uncovered(pc.m0, pc.m1, rows), b_hat = uncovered(pc.n0, pc.n1, cols);
+            const uint64_t c = std::max(std::max(cost_dl(a_hat, b_hat, kk, d, o.b_in, false), cost_ul(a, b, d, o.b_out)),
+                                        cost_comp(a, b, kk, d));
+            const u128 cand = r.load[k] + c;
+            if (!found || cand < best_cand) { found = true; best_cand = cand; best_cost = c; best_dev = k; }
+        }
+        if (!found) return CLEAVE_E_INFEASIBLE;
+        pc.dev = best_dev;
+        pc.cost_ns = best_cost;
+        r.load[best_dev] += best_cost;
+        r.held[best_dev].push_back(pc.id);
+    }
+
+    for (uint32_t f : F) p.tasks[f].flags |= CLEAVE_TASK_SUPERSEDED;
+    for (auto& kv : rounds) p.dead[kv.first] = kv.second.dead;
+    p.tasks.insert(p.tasks.end(), pieces.begin(), pieces.end());
+    p.dropped.resize(p.tasks.size(), 0);
+    build_tiles(p, *first_new);
+    return 0;
+}
+
+// ---- exec work list -----------------------------------------------------------------------------
+// A task is cut into tiles of 128 rows x w columns, w <= 256 chosen so the column tiles are balanced
+// and 16-aligned.  Tiles are ordered so that tiles running at the same time share operand panels in
+// L2: by GEMM, K-range, band of 2048 rows, then column, then row.
+void build_tiles(cleave_plan_s& p, uint32_t first_task) {
+    const uint32_t kBandRows = 2048;
+    const size_t begin = p.tiles.size();
+    p.task_ntiles.resize(p.tasks.size(), 0);
+    for (uint32_t id = first_task; id < p.tasks.size(); ++id) {
+        const cleave_task_t& t = p.tasks[id];
+        const cleave_gemm_t& g = p.gemms[t.gemm];
+        const uint32_t alpha = t.m1 - t.m0, beta = t.n1 - t.n0;
+        if ((t.k0 % 64) || ((t.k1 % 64) && t.k1 != g.K) || (g.transA && (t.m0 % 8)) || (!g.transB && (t.n0 % 8)) ||
+            (g.lda % 8) || (g.ldb % 8))
+            p.exec_unsupported = 1;
+        const uint32_t nt0 = (uint32_t)cdiv(beta, 256);
+        const uint32_t w = (uint32_t)(cdiv(cdiv(beta, nt0), 16) * 16);
+        const uint32_t nt = (uint32_t)cdiv(beta, w), mt = (uint32_t)cdiv(alpha, 128);
+        p.task_ntiles[id] = nt * mt;
+        for (uint32_t ti = 0; ti < mt; ++ti)
+            for (uint32_t tj = 0; tj < nt; ++tj) {
+                TileDesc d;
+                std::memset(&d, 0, sizeof d);
+                d.task = id; d.gemm = t.gemm;
+                d.flags = TILE_VALID | (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN);
+                d.rows = std::min(128u, alpha - ti * 128);
+                d.cols = std::min(w, beta - tj * w);
+                d.n_mma = (d.cols + 15) / 16 * 16;
+                d.m_row = t.m0 + ti * 128;
+                d.n_col = t.n0 + tj * w;
+                d.k0 = t.k0; d.k1 = t.k1;
+                d.ld = beta;
+                d.out_off = t.part_off + (uint64_t)ti * 128 * beta + (uint64_t)tj * w;
+                p.tiles.push_back(d);
+            }
+    }
+    std::stable_sort(p.tiles.begin() + begin, p.tiles.end(), [&](const TileDesc& a, const TileDesc& b) {
+        if (a.gemm != b.gemm) return a.gemm < b.gemm;
+        if (a.k0 != b.k0) return a.k0 < b.k0;
+        const uint32_t ba = a.m_row / kBandRows, bb = b.m_row / kBandRows;
+        if (ba != bb) return ba < bb;
+        if (a.n_col != b.n_col) return a.n_col < b.n_col;
+        return a.m_row < b.m_row;
+    });
+}
+
+// ---- assembly work list ---------------------------------------------------------------------------
+// All row / column boundaries of a GEMM's original tasks cut C into cells; in a cell every K-slice is
+// served by exactly one task.  Neighbouring cells served by the same tasks are merged again, then
+// the rectangles are cut into items of whole rows of roughly 16K outputs each.
+int build_assembly(cleave_plan_s& p) {
+    p.asm_items.clear(); p.asm_refs.clear(); p.asm_groups.clear();
+    std::vector<uint32_t> first_item, gemm_sp;       // per GEMM: first item, launch class
+    std::vector<std::vector<uint32_t>> by_gemm(p.gemms.size());
+    for (uint32_t id = 0; id < p.n_original; ++id) by_gemm[p.tasks[id].gemm].push_back(id);
+    for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
+        first_item.push_back((uint32_t)p.asm_items.size());
+        const cleave_gemm_t& g = p.gemms[gi];
+        const uint32_t S = p.ksplit[gi];
+        std::vector<uint32_t> rc, cc;
+        for (uint32_t id : by_gemm[gi]) {
+            const cleave_task_t& t = p.tasks[id];
+            rc.push_back(t.m0); rc.push_back(t.m1); cc.push_back(t.n0); cc.push_back(t.n1);
+        }
+        std::sort(rc.begin(), rc.end()); rc.erase(std::unique(rc.begin(), rc.end()), rc.end());
+        std::sort(cc.begin(), cc.end()); cc.erase(std::unique(cc.begin(), cc.end()), cc.end());
+        const size_t nr = rc.size() - 1, nc = cc.size() - 1;
+        std::vector<uint32_t> cell(nr * nc * S, UINT32_MAX);
+        for (uint32_t id : by_gemm[gi]) {
+            const cleave_task_t& t = p.tasks[id];
+            if (t.kslice >= S) return CLEAVE_E_INVAL;
+            const size_t r0 = std::lower_bound(rc.begin(), rc.end(), t.m0) - rc.begin();
+            const size_t r1 = std::lower_bound(rc.begin(), rc.end(), t.m1) - rc.begin();
+            const size_t c0 = std::lower_bound(cc.begin(), cc.end(), t.n0) - cc.begin();
+            const size_t c1 = std::lower_bound(cc.begin(), cc.end(), t.n1) - cc.begin();
+            for (size_t r = r0; r < r1; ++r)
+                for (size_t c = c0; c < c1; ++c) cell[(r * nc + c) * S + t.kslice] = id;
+        }
+        for (uint32_t x : cell) if (x == UINT32_MAX) return CLEAVE_E_INVAL;   // not a tiling
+        (void)g;
+        // merge: horizontal runs per cell row, then vertical runs of identical (columns, tasks)
+        struct Seg { uint32_t i0, i1, j0, j1; std::vector<uint32_t> tasks; };
+        std::vector<Seg> open, done;
+        for (size_t r = 0; r < nr; ++r) {
+            std::vector<Seg> row;
+            for (size_t c = 0; c < nc; ++c) {
+                std::vector<uint32_t> ts(cell.begin() + (r * nc + c) * S, cell.begin() + (r * nc + c + 1) * S);
+                if (!row.empty() && row.back().tasks == ts && row.back().j1 == cc[c]) row.back().j1 = cc[c + 1];
+                else row.push_back(Seg{rc[r], rc[r + 1], cc[c], cc[c + 1], ts});
+            }
+            std::vector<Seg> next_open;
+            for (Seg& s : row) {
+                bool merged = false;
+                for (Seg& o : open)
+                    if (o.i1 == s.i0 && o.j0 == s.j0 && o.j1 == s.j1 && o.tasks == s.tasks) { o.i1 = s.i1; next_open.push_back(o); o.i1 = UINT32_MAX; merged = true; break; }
+                if (!merged) next_open.push_back(s);
+            }
+            for (Seg& o : open) if (o.i1 != UINT32_MAX) done.push_back(o);
+            open.swap(next_open);
+        }
+        for (Seg& o : open) done.push_back(o);
+        std::sort(done.begin(), done.end(), [](const Seg& a, const Seg& b) { return a.i0 != b.i0 ? a.i0 < b.i0 : a.j0 < b.j0; });
+
+        bool vec = (g.N % 4 == 0);
+        for (const Seg& s : done) {
+            const uint32_t ncols = s.j1 - s.j0;
+            const uint32_t rows_per = std::max(1u, 16384u / ncols);
+            if (s.j0 % 4 || ncols % 4) vec = false;
+            for (uint32_t i = s.i0; i < s.i1; i += rows_per) {
+                AsmItem it;
+                it.gemm = gi; it.i0 = i; it.nrows = std::min(rows_per, s.i1 - i);
+                it.j0 = s.j0; it.ncols = ncols; it.ref0 = (uint32_t)p.asm_refs.size(); it.nslices = S; it.pad = 0;
+                for (uint32_t sl = 0; sl < S; ++sl) {
+                    const cleave_task_t& t = p.tasks[s.tasks[sl]];
+                    AsmRef r;
+                    r.ld = t.n1 - t.n0;
+                    r.off = t.part_off + (uint64_t)(i - t.m0) * r.ld + (s.j0 - t.n0);
+                    r.task = t.id;
+                    if (r.off % 4 || r.ld % 4) vec = false;
+                    p.asm_refs.push_back(r);
+                }
+                p.asm_items.push_back(it);
+            }
+        }
+        uint32_t sp = 1;
+        while (sp < S) sp *= 2;
+        gemm_sp.push_back(vec ? sp : 0u);
+    }
+    first_item.push_back((uint32_t)p.asm_items.size());
+    // one launch per class: reorder the items so that each class is contiguous (GEMM order inside)
+    std::vector<AsmItem> sorted;
+    sorted.reserve(p.asm_items.size());
+    for (uint32_t cls : {1u, 2u, 4u, 8u, 16u, 32u, 0u}) {
+        const uint32_t item0 = (uint32_t)sorted.size();
+        for (uint32_t gi = 0; gi < p.gemms.size(); ++gi)
+            if (gemm_sp[gi] == cls)
+                sorted.insert(sorted.end(), p.asm_items.begin() + first_item[gi], p.asm_items.begin() + first_item[gi + 1]);
+        if (sorted.size() > item0) p.asm_groups.push_back({cls, item0, (uint32_t)sorted.size() - item0});
+    }
+    p.asm_items.swap(sorted);
+    return 0;
+}
+
+}  // namespace cleave

@@ -1,0 +1,174 @@
+"""Parity of the CUDA path against the oracle, through the C ABI.  Needs a B200."""
+import numpy as np
+import pytest
+
+import cleave_inputs as ci
+from helpers import (GpuRun, assert_within_tolerance, lib_plan_for, oracle_operands, oracle_plan_for,
+                     task_matrix_lib, task_matrix_oracle)
+from oracle import check, numerics as nm
+from oracle.reissue import reissue as oracle_reissue
+
+pytestmark = pytest.mark.gpu
+
+
+def _custom_workload(tokens, projections, passes=("fwd", "dgrad", "wgrad"), n_devices=6, uniform=None, seed=0):
+    gemms, tensors = ci.projection_gemms(tokens, projections, passes)
+    return ci.Workload("custom", gemms, tensors, n_devices=n_devices, mem_range=(64 * ci.MB, 1 * ci.GB),
+                       uniform=uniform, seed=seed)
+
+
+def _run_and_compare_exact(w, opts=None, integer=True):
+    opts = opts or {}
+    ts = ci.make_tensors(w, integer=integer)
+    p, op = lib_plan_for(w, **opts), oracle_plan_for(w, **opts)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    A, B = oracle_operands(w, ts)
+    ref = nm.assemble(op, nm.execute(op, A, B))
+    run = GpuRun(w, ts, p)
+    run.exec()
+    run.assemble()
+    p.check_status()
+    out = run.results()
+    for gi, g in enumerate(w.gemms):
+        if integer:
+            assert np.array_equal(out[gi].astype(np.float64), ref[gi]), f"{g.name}: integer inputs must be exact"
+        else:
+            assert_within_tolerance(out[gi], ref[gi], nm.abs_bound(A[gi], B[gi]), what=g.name)
+    done = p.done_counts()
+    assert all(done[i] == p.task_num_tiles(i) for i in range(p.num_tasks))
+    return p, op, run, ref
+
+
+def test_config1_uniform_exact_and_gaussian():
+    w = ci.config(1)
+    _run_and_compare_exact(w, integer=True)
+    _run_and_compare_exact(w, integer=False)
+
+
+@pytest.mark.parametrize("passes", [("fwd",), ("dgrad",), ("wgrad",)])
+def test_each_operand_layout_exact(passes):
+    # several tiles per task, two K-slices, ragged last tile in every dimension
+    w = _custom_workload(648, [("p", 456, 328)], passes=passes, n_devices=5)
+    _run_and_compare_exact(w, dict(kslice_max=256))
+
+
+def test_ragged_uniform_grid_exact():
+    # block edges that are multiples of 8 but not of the tile; K tail 40 beyond a multiple of 64
+    w = _custom_workload(520, [("p", 424, 392)], uniform=(3, 2, 1))
+    w.n_devices = 0
+    _run_and_compare_exact(w)
+
+
+def test_wide_and_tall_tasks_exact():
+    # one device: a single task per K-slice, many 128 x 256 tiles, three K-slices
+    w = _custom_workload(1024, [("p", 832, 1280)], n_devices=1)
+    p, *_ = _run_and_compare_exact(w, dict(kslice_max=512))
+    assert max(p.ksplit(i) for i in range(3)) >= 2
+
+
+@pytest.mark.parametrize("cfg,scale", [(2, 4), (3, 8), (5, 16)])
+def test_scaled_configs_gaussian(cfg, scale):
+    w = ci.config(cfg, scale)
+    _run_and_compare_exact(w, integer=False)
+
+
+def test_scaled_config2_integer_exact():
+    _run_and_compare_exact(ci.config(2, 4), integer=True)
+
+
+def test_churn_reissue_equals_no_failure():
+    w = ci.config(4, 8)
+    ts = ci.make_tensors(w, integer=False)
+    p, op = lib_plan_for(w), oracle_plan_for(w)
+    A, B = oracle_operands(w, ts)
+    ref = nm.assemble(op, nm.execute(op, A, B))
+
+    base = GpuRun(w, ts, p)                  # no failure
+    base.exec(); base.assemble(); p.check_status()
+    good = base.results()
+
+    p2 = lib_plan_for(w)
+    failed = ci.make_failed_ids(p2.num_tasks, w.fail_frac, w.seed + 2)
+    p2.set_drops(failed)
+    run = GpuRun(w, ts, p2)                  # arena poisoned with NaN: a skipped block stays NaN
+    run.exec(); run.assemble()
+    assert p2.status() == -9                 # E_INCOMPLETE: bookkeeping knows what is missing
+    assert any(np.isnan(c).any() for c in run.results())
+    done = p2.done_counts()
+    assert all((done[i] == 0) == (i in set(failed.tolist())) for i in range(p2.num_tasks))
+
+    run.reissue(failed)                      # explicit failed list
+    new = oracle_reissue(op, failed)
+    assert np.array_equal(task_matrix_lib(p2), task_matrix_oracle(op))
+    run.assemble()
+    assert p2.status() == 0
+    out = run.results()
+    for gi, g in enumerate(w.gemms):
+        assert np.array_equal(out[gi], good[gi]), f"{g.name}: reissued result differs from the no-failure result"
+        assert_within_tolerance(out[gi], ref[gi], nm.abs_bound(A[gi], B[gi]), what=g.name)
+
+    # second wave, found by the bookkeeping itself (n = 0): drop some replacement tasks and re-run all
+    again = [t.id for t in new[::4]]
+    p2.set_drops(again)
+    run.partials.fill_(float("nan"))
+    run.exec(); run.assemble()
+    assert p2.status() == -9
+    run.reissue(None)
+    oracle_reissue(op, again)
+    assert np.array_equal(task_matrix_lib(p2), task_matrix_oracle(op))
+    run.assemble()
+    assert p2.status() == 0
+    out = run.results()
+    for gi in range(len(w.gemms)):
+        assert np.array_equal(out[gi], good[gi])
+
+
+@pytest.mark.parametrize("S", [1, 2, 3, 4, 5, 8, 13])
+def test_assembly_bit_exact_vs_fp32_tree(S):
+    """Random fp32 partials (not products): the assembly kernel must reproduce the balanced
+    pairwise tree bit for bit."""
+    import torch
+    w = _custom_workload(384, [("p", 128 * S, 320)], passes=("fwd",), n_devices=7, seed=S)
+    opts = dict(ksplit=S, kslice_max=0, ksplit_cap=32)
+    p, op = lib_plan_for(w, **opts), oracle_plan_for(w, **opts)
+    assert p.ksplit(0) == S
+    rng = np.random.default_rng(S)
+    arena = (rng.standard_normal(op.arena_elems) * 10.0 ** rng.integers(-3, 4, op.arena_elems)).astype(np.float32)
+    ref = nm.assemble(op, arena, dtype=np.float32)[0]
+    g = w.gemms[0]
+    C = torch.zeros((g.M, g.N), dtype=torch.float32, device="cuda:0")
+    part = torch.from_numpy(arena).cuda()
+    p.assemble(part, [C])
+    assert p.status() == -9                  # nothing was executed: bookkeeping says incomplete ...
+    out = C.cpu().numpy()
+    assert np.array_equal(out.view(np.uint32), ref.view(np.uint32))   # ... the sums are exact all the same
+
+
+def test_assembly_scalar_path_bit_exact():
+    import torch
+    gemms, tensors = ci.projection_gemms(50, [("p", 64, 45)], ("fwd",))      # N = 45: no float4 alignment
+    w = ci.Workload("odd", gemms, tensors, uniform=(3, 2, 1))
+    from oracle.plan import Opts, plan_uniform
+    import paper_2512_22142_b200 as cl
+    p = cl.plan_uniform(w.gemms, 3, 2, 1)
+    op = oracle_plan_for(w)
+    rng = np.random.default_rng(0)
+    arena = rng.standard_normal(op.arena_elems).astype(np.float32)
+    ref = nm.assemble(op, arena, dtype=np.float32)[0]
+    C = torch.zeros((50, 45), dtype=torch.float32, device="cuda:0")
+    p.assemble(torch.from_numpy(arena).cuda(), [C])
+    torch.cuda.synchronize()
+    assert np.array_equal(C.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
+def test_unsupported_alignment_is_rejected():
+    import torch
+    import paper_2512_22142_b200 as cl
+    gemms, tensors = ci.projection_gemms(64, [("p", 200, 64)], ("fwd",))     # K = 200 in 2 slices of 100
+    p = cl.plan_uniform(gemms, 1, 1, 2)
+    x = torch.zeros(64, 200, dtype=torch.bfloat16, device="cuda:0")
+    wt = torch.zeros(200, 64, dtype=torch.bfloat16, device="cuda:0")
+    part = torch.zeros(p.arena_elems, dtype=torch.float32, device="cuda:0")
+    with pytest.raises(cl.CleaveError) as e:
+        p.exec([x], [wt], part)
+    assert e.value.code == -2
