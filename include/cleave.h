@@ -171,8 +171,8 @@ CLEAVE_API int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t
  * tasks run at the next cleave_exec.  Works without a CUDA device. */
 CLEAVE_API int cleave_replan(cleave_plan_t* p, const uint32_t* failed, uint32_t n, uint32_t* first_new);
 
-/* Synchronises `stream` and returns the device status: 0, E_TIMEOUT, E_BOUNDS or E_INCOMPLETE
- * (the most severe seen since the last cleave_exec), or E_CUDA. */
+/* Synchronises `stream` and returns the device status: 0, E_TIMEOUT or E_BOUNDS (sticky since
+ * the last cleave_exec), E_INCOMPLETE (verdict of the latest cleave_assemble), or E_CUDA. */
 CLEAVE_API int cleave_status(cleave_plan_t* p, void* stream);
 
 /* Number of finished tiles of each task, copied to host (synchronises the stream).

@@ -386,6 +386,8 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
 // -------------------------------------------------------------------------------------------------
 // bookkeeping kernels
 // -------------------------------------------------------------------------------------------------
+__global__ void clear_status_bits_kernel(unsigned int* status, unsigned int mask) { *status &= ~mask; }
+
 __global__ void check_done_kernel(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
                                   uint32_t n_tasks, unsigned int* status) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -527,7 +529,9 @@ cudaError_t launch_exec(uint32_t grid, const TileDesc* tiles, uint32_t tile_end,
 
 cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles, uint32_t n_tasks,
                               unsigned int* status, cudaStream_t st) {
-    if (!n_tasks) return cudaSuccess;
+    // the verdict belongs to this assembly: forget the one of an earlier call
+    clear_status_bits_kernel<<<1, 1, 0, st>>>(status, STATUS_INCOMPLETE);
+    if (!n_tasks) return cudaGetLastError();
     check_done_kernel<<<(n_tasks + 255) / 256, 256, 0, st>>>(tasks, done, ntiles, n_tasks, status);
     return cudaGetLastError();
 }
