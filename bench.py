@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the Cleave hot path on B200: decomposed GEMM + assembly throughput per step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 3]
+
+A step is one pass of the path over one batch of synthetic input: queue arming, the grouped
+sub-GEMM execution of every task of every GEMM of the layer, and the assembly of the K-split
+partial blocks into the GEMM results.  The plan is made once before the loop (the paper solves the
+schedule once per device set and reuses it); its time and the churn path (drop 10 % of the tasks,
+re-plan, reissue, re-assemble) are measured separately and reported inside `config`.
+
+One JSON line is printed by rank 0.  With --gpus N > 1 (launched through torch.distributed.run)
+every rank runs an independent replica of the same workload on its own GPU: the path has no
+inter-GPU exchange step, so there is no collective on the data path ("replicas only").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decomposed GEMM+assembly TFLOP/s and % of B200 dense BF16 peak, per step"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# --------------------------------------------------------------------------------------------------
+REASON_BITS = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+               0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+
+class ClockSampler:
+    def __init__(self, device_index: int):
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for b, name in REASON_BITS.items():
+                    if bits & b:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------------
+# the oracle on the host cores (reported baseline / --impl reference)
+# --------------------------------------------------------------------------------------------------
+def oracle_block_groups(w, opts):
+    """The oracle's own plan of the workload, its tasks grouped by output rectangle (all K-slices
+    of one block), in a seeded random order."""
+    import numpy as np
+    import cleave_inputs as ci
+    from oracle.cost import devices_from_array
+    from oracle.plan import Gemm, Opts, plan, plan_uniform
+    gemms = [Gemm(g.M, g.N, g.K, g.transA, g.transB) for g in w.gemms]
+    t0 = time.perf_counter()
+    devs = ci.workload_devices(w)
+    op = plan_uniform(gemms, *w.uniform, Opts(**opts)) if devs is None else plan(gemms, devices_from_array(devs), Opts(**opts))
+    plan_s = time.perf_counter() - t0
+    groups = {}
+    for t in op.tasks:
+        groups.setdefault((t.gemm, t.m0, t.m1, t.n0, t.n1), []).append(t)
+    keys = sorted(groups)
+    order = np.random.default_rng(w.seed + 3).permutation(len(keys))
+    return op, [groups[keys[i]] for i in order], plan_s
+
+
+def oracle_run_groups(w, bits, groups):
+    """fp64 sub-GEMMs of every task of the groups plus the tree-sum of each block's K-slices."""
+    from oracle import numerics as nm
+    flops = 0
+    for tasks in groups:
+        g = w.gemms[tasks[0].gemm]
+        parts = [nm.sub_gemm_from_bits(t, g.transA, g.transB, bits[g.a_key], bits[g.b_key])
+                 for t in sorted(tasks, key=lambda t: t.kslice)]
+        nm.tree_sum(parts)
+        flops += sum(2 * t.alpha * t.beta * t.kappa for t in tasks)
+    return flops
+
+
+def blas_threads():
+    try:
+        import threadpoolctl
+        n = [i["num_threads"] for i in threadpoolctl.threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def cpu_baseline(w, tensors, opts, budget_s=15.0):
+    import cleave_inputs as ci
+    bits = {k: ci.bf16_bits(t) for k, t in tensors.items()}
+    op, groups, plan_s = oracle_block_groups(w, opts)
+    t0 = time.perf_counter()
+    flops, n = 0, 0
+    for grp in groups:
+        flops += oracle_run_groups(w, bits, [grp])
+        n += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{n} of {len(groups)} output blocks (all K-slices each, seeded random order) of {w.name}: "
+                      f"fp64 sub-GEMMs + tree assembly, {flops / 1e12:.3f} TFLOP in {dt:.1f} s; "
+                      f"oracle plan of the full workload took {plan_s:.2f} s (not in the rate)",
+            "host_cores_available": len(os.sched_getaffinity(0))}
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, on the host cores; each step is a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import cleave_inputs as ci
+    w = ci.config(args.config)
+    tensors = ci.make_tensors(w)
+    bits = {k: ci.bf16_bits(t) for k, t in tensors.items()}
+    op, groups, plan_s = oracle_block_groups(w, {})
+    # size a step: calibrate on a few blocks, then fix the number of blocks per step
+    t0 = time.perf_counter()
+    oracle_run_groups(w, bits, groups[:4])
+    per_block = (time.perf_counter() - t0) / 4
+    step_budget = min(2.0, 90.0 / (args.steps + args.warmup))
+    per_step = max(1, min(len(groups) // (args.steps + args.warmup), int(step_budget / max(per_block, 1e-6))))
+    cursor = 0
+    for _ in range(args.warmup):
+        oracle_run_groups(w, bits, groups[cursor:cursor + per_step]); cursor += per_step
+    flops, t0 = 0, time.perf_counter()
+    for _ in range(args.steps):
+        flops += oracle_run_groups(w, bits, groups[cursor:cursor + per_step]); cursor += per_step
+    dt = time.perf_counter() - t0
+    value = flops / dt / 1e12
+    sample = (f"each step = {per_step} of {len(groups)} output blocks (all K-slices each) of {w.name}: fp64 sub-GEMMs + "
+              f"tree assembly on the host cores")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "gemms": len(w.gemms), "devices": w.n_devices, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# the CUDA path
+# --------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    import cleave_inputs as ci
+    import paper_2512_22142_b200 as cl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = ci.config(args.config)
+    opts = {}
+    if args.kslice_max is not None:
+        opts["kslice_max"] = args.kslice_max
+    t0 = time.perf_counter()
+    tensors = ci.make_tensors(w, pin=True)
+    gen_s = time.perf_counter() - t0
+    devs = ci.workload_devices(w)
+    t0 = time.perf_counter()
+    plan = cl.plan_uniform(w.gemms, *w.uniform, cl.default_opts(**opts)) if devs is None else cl.plan(w.gemms, devs, cl.default_opts(**opts))
+    plan_ms = (time.perf_counter() - t0) * 1e3
+
+    d_tensors = {k: t.to(dev) for k, t in tensors.items()}
+    A = [d_tensors[g.a_key] for g in w.gemms]
+    B = [d_tensors[g.b_key] for g in w.gemms]
+    partials = torch.empty(plan.arena_elems, dtype=torch.float32, device=dev)
+    C = [torch.empty((g.M, g.N), dtype=torch.float32, device=dev) for g in w.gemms]
+    flops = float(w.flops)
+    S = [plan.ksplit(i) for i in range(len(w.gemms))]
+    asm_bytes = float(sum((S[i] + 1) * g.M * g.N * 4 for i, g in enumerate(w.gemms)))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident steps -------------------------------------------------------------------
+    for _ in range(args.warmup):
+        plan.exec(A, B, partials)
+        plan.assemble(partials, C)
+    plan.check_status()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    if sampler:
+        sampler.start()
+    begin, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    begin.record()
+    for s in range(args.steps):
+        ev[s][0].record()
+        plan.exec(A, B, partials)
+        ev[s][1].record()
+        plan.assemble(partials, C)
+        ev[s][2].record()
+    end.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    plan.check_status()
+    total_ms = max_over_ranks(begin.elapsed_time(end))
+    exec_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    asm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    ms_per_step = total_ms / args.steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----------------
+    host_C = [torch.empty((g.M, g.N), dtype=torch.float32).pin_memory() for g in w.gemms]
+    h2d = sum(t.numel() * 2 for t in tensors.values())
+    d2h = sum(c.numel() * 4 for c in host_C)
+
+    def e2e_step():
+        for k, t in tensors.items():
+            d_tensors[k].copy_(t, non_blocking=True)
+        plan.exec(A, B, partials)
+        plan.assemble(partials, C)
+        for hc, c in zip(host_C, C):
+            hc.copy_(c, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    b2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b2.record()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e2.record()
+    barrier()
+    e2e_ms = max_over_ranks(b2.elapsed_time(e2)) / args.e2e_steps
+    e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
+    checksum = float(host_C[0][0, :8].double().sum())
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- churn path (rank 0, once): drop 10 %, execute, re-plan + reissue, re-assemble ------------------
+    churn = None
+    if devs is not None and not args.no_churn:
+        p2 = cl.plan(w.gemms, devs, cl.default_opts(**opts))
+        failed = ci.make_failed_ids(p2.num_tasks, 0.10, w.seed + 2)
+        p2.set_drops(failed)
+        p2.exec(A, B, partials)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        c0, c1, c2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        c0.record()
+        p2.reissue(failed, A, B, partials)
+        host_ms = (time.perf_counter() - t0) * 1e3
+        c1.record()
+        p2.assemble(partials, C)
+        c2.record()
+        torch.cuda.synchronize()
+        churn = {"failed_tasks": int(len(failed)), "reissued_tasks": int(p2.num_tasks - p2.num_original),
+                 "reissue_host_ms": host_ms, "reissue_device_ms": c0.elapsed_time(c1), "reassemble_ms": c1.elapsed_time(c2),
+                 "status": p2.status()}
+        p2.close()
+
+    peaks, peak_kind = load_peaks()
+    exec_tflops = flops / (exec_ms * 1e-3) / 1e12
+    asm_gbs = asm_bytes / (asm_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": w.name, "gemms": len(w.gemms), "devices": w.n_devices, "tasks": plan.num_tasks,
+            "tiles": plan.num_tiles, "flop_per_step": flops, "ksplit": S, "arena_GB": plan.arena_elems * 4 / 1e9,
+            "parallelism": "replicas only" if world > 1 else "1 GPU",
+            "l2": "not flushed; operands + arena + outputs per step (~%.1f GB) far exceed the 126 MB L2" %
+                  ((h2d + plan.arena_elems * 4 + d2h) / 1e9),
+            "plan_ms_host": plan_ms, "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
+            "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
+            "pct_of_measured_sustained_bf16": 100 * value / world / peaks["bf16_tflops_sustained"],
+            "churn": churn, "e2e_ms_per_step": e2e_ms, "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
+        },
+        "roofline": {"kernel": "exec_kernel", "bound": "tensor", "achieved": exec_tflops, "peak": peaks["bf16_tflops_sustained"],
+                     "unit": "TFLOP/s", "frac": exec_tflops / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "peak_kind": f"{peak_kind}, sustained cuBLAS bf16 (kernel timed inside a long step)",
+                     "frac_of_burst": exec_tflops / peaks["bf16_tflops"], "frac_of_nominal": exec_tflops / NOMINAL_BF16_TFLOPS},
+        "roofline_assemble": {"kernel": "assemble_vec_kernel", "bound": "hbm", "achieved": asm_gbs, "peak": peaks["hbm_gbs"],
+                              "unit": "GB/s", "frac": asm_gbs / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind,
+                              "frac_of_nominal": asm_gbs / NOMINAL_HBM_GBS, "algorithmic_bytes": asm_bytes},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": plan.num_launches * args.steps,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(w, tensors, opts, args.cpu_budget)
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3, help="workload: 1..5 (3 = Llama-7B-shaped layer, the headline)")
+    ap.add_argument("--kslice-max", type=int, default=None, help="deepest K-slice (planner option); default 4096")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-churn", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -125,6 +125,8 @@ CLEAVE_API uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm);  
 CLEAVE_API uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm);  /* modelled, max load  */
 CLEAVE_API uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm);     /* water-fill level    */
 CLEAVE_API uint32_t cleave_plan_num_tiles(const cleave_plan_t* p);        /* work units of the exec kernel  */
+CLEAVE_API uint32_t cleave_plan_num_launches(const cleave_plan_t* p);     /* kernels launched by one
+                                                  cleave_exec followed by one cleave_assemble    */
 
 /* Host-made failures (Section 3.2, "Device departures are detected via disconnect events"): the
  * listed tasks are skipped by every later cleave_exec / cleave_reissue launch, as if their device

@@ -37,6 +37,14 @@ def sub_gemm(t: Task, A: np.ndarray, B: np.ndarray) -> np.ndarray:
     return A[t.m0:t.m1, t.k0:t.k1] @ B[t.k0:t.k1, t.n0:t.n1]
 
 
+def sub_gemm_from_bits(t: Task, transA: int, transB: int, a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
+    """Same block as `sub_gemm`, starting from the stored bf16 bit patterns: only the task's own
+    rows of A and columns of B are widened (what a device would be sent)."""
+    a = a_bits[t.k0:t.k1, t.m0:t.m1].T if transA else a_bits[t.m0:t.m1, t.k0:t.k1]
+    b = b_bits[t.n0:t.n1, t.k0:t.k1].T if transB else b_bits[t.k0:t.k1, t.n0:t.n1]
+    return bf16_bits_to_f64(np.ascontiguousarray(a)) @ bf16_bits_to_f64(np.ascontiguousarray(b))
+
+
 def execute(plan: Plan, A: Sequence[np.ndarray], B: Sequence[np.ndarray],
             task_ids=None, arena: np.ndarray = None, dropped=()) -> np.ndarray:
     """Runs tasks (all live ones by default) and writes each block, row-major with leading

@@ -45,6 +45,7 @@ _sig = {
     "cleave_plan_makespan_ns": (_u64, [_vp, _u32]),
     "cleave_plan_tstar_ns": (_u64, [_vp, _u32]),
     "cleave_plan_num_tiles": (_u32, [_vp]),
+    "cleave_plan_num_launches": (_u32, [_vp]),
     "cleave_set_drops": (_i, [_vp, _vp, _u32]),
     "cleave_exec": (_i, [_vp, _vp, _vp, _vp, _vp]),
     "cleave_assemble": (_i, [_vp, _vp, _vp, _vp]),
@@ -138,6 +139,10 @@ class Plan:
     @property
     def num_tiles(self) -> int:
         return lib.cleave_plan_num_tiles(self._h)
+
+    @property
+    def num_launches(self) -> int:
+        return lib.cleave_plan_num_launches(self._h)
 
     @property
     def arena_elems(self) -> int:

@@ -274,6 +274,8 @@ uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm) { return (p &
 uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->makespan.size()) ? p->makespan[gemm] : 0; }
 uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->tstar.size()) ? p->tstar[gemm] : 0; }
 uint32_t cleave_plan_num_tiles(const cleave_plan_t* p) { return p ? (uint32_t)p->tiles.size() : 0; }
+// exec: arm + grouped GEMM; assemble: clear verdict + bookkeeping check + one kernel per slice-count class
+uint32_t cleave_plan_num_launches(const cleave_plan_t* p) { return p ? 4u + (uint32_t)p->asm_groups.size() : 0; }
 uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task) { return (p && task < p->task_ntiles.size()) ? p->task_ntiles[task] : 0; }
 
 int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t n) {

@@ -104,3 +104,15 @@ def test_sample_entries():
     rows, cols = np.array([0, 3, 9]), np.array([8, 1, 4])
     c, bound = nm.sample_entries(A, B, rows, cols)
     assert np.allclose(c, (A @ B)[rows, cols]) and np.allclose(bound, (np.abs(A) @ np.abs(B))[rows, cols])
+
+
+def test_sub_gemm_from_bits_matches_sub_gemm():
+    w = ci.config(2, scale=16)
+    ts = ci.make_tensors(w)
+    p = plan([Gemm(g.M, g.N, g.K, g.transA, g.transB) for g in w.gemms],
+             devices_from_array(ci.workload_devices(w)), Opts(gran_m=32, gran_n=32, gran_k=32, kslice_max=64))
+    for t in p.tasks[::7]:
+        g = w.gemms[t.gemm]
+        a_bits, b_bits = ci.bf16_bits(ts[g.a_key]), ci.bf16_bits(ts[g.b_key])
+        full = nm.sub_gemm(t, nm.op_a(nm.bf16_bits_to_f64(a_bits), g.transA), nm.op_b(nm.bf16_bits_to_f64(b_bits), g.transB))
+        assert np.array_equal(nm.sub_gemm_from_bits(t, g.transA, g.transB, a_bits, b_bits), full)
