@@ -376,7 +376,7 @@ int cleave_done_counts(cleave_plan_t* p, uint32_t* done, void* stream) {
     std::fill(done, done + n, 0u);
     CU_TRY(cudaMemcpyAsync(done, p->dev->done, have * 4, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
-    for (size_t i = 0; i < have; ++i) done[i] /= kEpiWarps;     // the kernel counts once per epilogue warp
+    for (size_t i = 0; i < have; ++i) done[i] /= kEpiWarpsPerGroup;   // the kernel counts once per epilogue warp
     return 0;
 }
 

@@ -5,8 +5,8 @@
 //   exec_kernel         persistent grouped GEMM: one CTA per SM walks the tile list through a
 //                       device-side ticket; TMA loads of 64x64 bf16 boxes into 128-byte-swizzled
 //                       shared memory, tcgen05 MMA (128 x N x 16, bf16 -> fp32) accumulating in
-//                       tensor memory, epilogue warps copy the accumulator to the task's packed
-//                       partial block and count the tile in the task's bookkeeping word
+//                       tensor memory, epilogue warps copy the accumulators to the task's packed
+//                       partial block and count each 128-row half-tile in the task's bookkeeping word
 //   check_done_kernel   flags E_INCOMPLETE if a live task has unfinished tiles
 //   assemble_kernel     fixed-order sum of the K-slices' partial blocks into C
 //   collect_failed_kernel  lists the live tasks whose bookkeeping shows unfinished tiles
@@ -165,11 +165,17 @@ __global__ void arm_queue_kernel(TileDesc* tiles, uint32_t tile_begin, uint32_t 
 // -------------------------------------------------------------------------------------------------
 // exec_kernel
 // -------------------------------------------------------------------------------------------------
+// Work unit: a tile of up to 256 rows x up to 256 columns of one task over the task's K-range.  The
+// rows are two halves of 128 (one MMA each per 16-deep K step) that share the B stage in shared
+// memory, so a 256-row tile moves a third fewer operand bytes per FLOP than two 128-row tiles.
+// Tensor memory holds two accumulator slots of 256 columns: a tall tile uses both (half h in slot
+// h), a tile of at most 128 rows uses one, alternating, so consecutive short tiles double-buffer.
+// Epilogue group g (four warps) drains slot g.
 struct __align__(16) ExecShared {
     uint64_t full[kStages];        // TMA bytes of a stage have landed
     uint64_t empty[kStages];       // the MMAs reading a stage have completed
-    uint64_t acc_full[kAccStages]; // an accumulator holds a finished tile
-    uint64_t acc_empty[kAccStages];// the epilogue has copied an accumulator out
+    uint64_t acc_full[kAccSlots];  // an accumulator slot holds a finished half-tile
+    uint64_t acc_empty[kAccSlots]; // the epilogue has copied an accumulator slot out
     uint64_t sched_full[kSchedSlots];
     uint64_t sched_empty[kSchedSlots];
     uint64_t drain;                // all MMAs completed (teardown)
@@ -191,7 +197,7 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh.full[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1); }
-        for (int a = 0; a < kAccStages; ++a) { mbar_init(smem_u32(&sh.acc_full[a]), 1); mbar_init(smem_u32(&sh.acc_empty[a]), kEpiWarps); }
+        for (int a = 0; a < kAccSlots; ++a) { mbar_init(smem_u32(&sh.acc_full[a]), 1); mbar_init(smem_u32(&sh.acc_empty[a]), kEpiWarpsPerGroup); }
         for (int q = 0; q < kSchedSlots; ++q) { mbar_init(smem_u32(&sh.sched_full[q]), 1); mbar_init(smem_u32(&sh.sched_empty[q]), 2 + kEpiWarps); }
         mbar_init(smem_u32(&sh.drain), 1);
         sh.abort_flag = 0;
@@ -227,46 +233,51 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
             }
         }
     } else if (warp == kTmaWarp) {
-        // ---- producer: TMA loads of the A and B sub-tiles of every K-block -------------------------
-        if (lane == 0) {
-            uint32_t it = 0, issued = 0, last_gemm = 0xFFFFFFFFu;
-            bool ok = true;
-            for (uint32_t i = 0; ok; ++i) {
-                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-                if (!mbar_wait(smem_u32(&sh.sched_full[q]), par, abort_flag, status)) break;
-                const TileDesc d = sh.slot[q];
-                mbar_arrive(smem_u32(&sh.sched_empty[q]));
-                if (d.flags & TILE_END) break;
-                const CUtensorMap* map_a = maps + 2 * d.gemm;
-                const CUtensorMap* map_b = map_a + 1;
-                if (d.gemm != last_gemm) { tensormap_acquire(map_a); tensormap_acquire(map_b); last_gemm = d.gemm; }
-                const bool a_mn = d.flags & TILE_A_MN, b_mn = d.flags & TILE_B_MN;   // M- / N-contiguous operand
-                const uint32_t nsub_a = d.rows > kSubRows ? 2u : 1u;
-                const uint32_t nsub_b = (d.n_mma + kSubRows - 1) / kSubRows;
-                const uint32_t tx = (nsub_a + nsub_b) * kSubBytes;
-                const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
-                for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
-                    const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
-                    if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, status)) { ok = false; break; }
-                    const uint32_t bar = smem_u32(&sh.full[s]);
-                    mbar_arrive_expect_tx(bar, tx);
-                    const uint32_t sa = stage_base + s * kStageBytes, sb = sa + kABytes;
-                    const int32_t k = (int32_t)(d.k0 + kb * kBlockK);
-                    for (uint32_t j = 0; j < nsub_a; ++j) {
-                        const int32_t m = (int32_t)(d.m_row + j * kSubRows);
-                        if (a_mn) tma_load_2d(sa + j * kSubBytes, map_a, bar, m, k);
-                        else      tma_load_2d(sa + j * kSubBytes, map_a, bar, k, m);
-                    }
-                    for (uint32_t j = 0; j < nsub_b; ++j) {
-                        const int32_t n = (int32_t)(d.n_col + j * kSubRows);
-                        if (b_mn) tma_load_2d(sb + j * kSubBytes, map_b, bar, n, k);
-                        else      tma_load_2d(sb + j * kSubBytes, map_b, bar, k, n);
-                    }
-                    ++issued;
+        // ---- producer: TMA loads of the A and B boxes of every K-block ------------------------------
+        // The whole warp walks the loop and lane j issues box j of a stage (up to 4 boxes of A, 4 of
+        // B): issued one after the other by a single thread, the boxes of a stage took longer to issue
+        // than the MMAs took to consume them.
+        uint32_t it = 0, issued = 0, last_gemm = 0xFFFFFFFFu;
+        bool ok = true;
+        for (uint32_t i = 0; ok; ++i) {
+            const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&sh.sched_full[q]), par, abort_flag, status))) break;
+            const TileDesc d = sh.slot[q];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.sched_empty[q]));
+            if (d.flags & TILE_END) break;
+            const CUtensorMap* map_a = maps + 2 * d.gemm;
+            const CUtensorMap* map_b = map_a + 1;
+            if (d.gemm != last_gemm) { tensormap_acquire(map_a); tensormap_acquire(map_b); last_gemm = d.gemm; }
+            const uint32_t nsub_a = (d.rows + kSubRows - 1) / kSubRows;      // stale rows beyond are never stored
+            const uint32_t nsub_b = (d.n_mma + kSubRows - 1) / kSubRows;
+            const uint32_t tx = (nsub_a + nsub_b) * kSubBytes;
+            const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
+            // this lane's box of a stage: operand, tensor map, offset in the stage, fixed coordinate
+            const bool is_a = lane < nsub_a, is_b = !is_a && lane < nsub_a + nsub_b;
+            const uint32_t j = is_a ? lane : lane - nsub_a;
+            const CUtensorMap* my_map = is_a ? map_a : map_b;
+            const bool my_mn = is_a ? (d.flags & TILE_A_MN) : (d.flags & TILE_B_MN);
+            const int32_t my_x = (int32_t)((is_a ? d.m_row : d.n_col) + j * kSubRows);
+            const uint32_t my_off = (is_a ? 0u : kABytes) + j * kSubBytes;
+            for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, status))) { ok = false; break; }
+                const uint32_t bar = smem_u32(&sh.full[s]);
+                if (lane == 0) mbar_arrive_expect_tx(bar, tx);
+                __syncwarp();
+                const int32_t k = (int32_t)(d.k0 + kb * kBlockK);
+                if (is_a || is_b) {
+                    const uint32_t dst = stage_base + s * kStageBytes + my_off;
+                    if (my_mn) tma_load_2d(dst, my_map, bar, my_x, k);
+                    else       tma_load_2d(dst, my_map, bar, k, my_x);
                 }
+                ++issued;
             }
-            // Wait for every copy still in flight before the CTA may exit (bounded).  A stage armed at
-            // iteration x completes phase (x / kStages) & 1 of its full barrier.
+        }
+        // Wait for every copy still in flight before the CTA may exit (bounded).  A stage armed at
+        // iteration x completes phase (x / kStages) & 1 of its full barrier.
+        if (lane == 0) {
             const uint32_t pending = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
             for (uint32_t x = it - pending; x < it; ++x) {
                 const uint64_t t0 = global_timer_ns();
@@ -277,7 +288,7 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
     } else if (warp == kMmaWarp) {
         // ---- MMA issuer ----------------------------------------------------------------------------
         if (lane == 0) {
-            uint32_t it = 0, acc_it = 0;
+            uint32_t it = 0, used0 = 0, used1 = 0, toggle = 0;     // used<s>: completed uses of accumulator slot s
             bool ok = true;
             for (uint32_t i = 0; ok; ++i) {
                 const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
@@ -293,10 +304,13 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
                 // of 16 is two such groups.
                 const uint32_t a_lbo = a_mn ? kSubBytes : 16u, a_step = a_mn ? 2048u : 32u;
                 const uint32_t b_lbo = b_mn ? kSubBytes : 16u, b_step = b_mn ? 2048u : 32u;
-                const uint32_t acc = acc_it % kAccStages, aph = (acc_it / kAccStages) & 1u;
-                if (!mbar_wait(smem_u32(&sh.acc_empty[acc]), aph ^ 1u, abort_flag, status)) break;
+                const bool tall = d.rows > kBlockM;
+                uint32_t slot0 = 0;
+                if (!tall) { slot0 = toggle; toggle ^= 1u; }
+                if (!mbar_wait(smem_u32(&sh.acc_empty[slot0]), ((slot0 ? used1 : used0) & 1u) ^ 1u, abort_flag, status)) break;
+                if (tall && !mbar_wait(smem_u32(&sh.acc_empty[1]), (used1 & 1u) ^ 1u, abort_flag, status)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                const uint32_t d0 = tmem_base + slot0 * kAccCols, d1 = tmem_base + kAccCols;
                 const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
                 for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                     const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
@@ -305,15 +319,17 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
                     const uint32_t sa = stage_base + s * kStageBytes, sb = sa + kABytes;
 #pragma unroll
                     for (uint32_t k16 = 0; k16 < kBlockK / 16; ++k16) {
-                        const uint64_t a_desc = smem_desc_sw128(sa + k16 * a_step, a_lbo, 1024u);
                         const uint64_t b_desc = smem_desc_sw128(sb + k16 * b_step, b_lbo, 1024u);
-                        umma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k16) != 0u);
+                        umma_bf16(d0, smem_desc_sw128(sa + k16 * a_step, a_lbo, 1024u), b_desc, idesc, (kb | k16) != 0u);
+                        if (tall)   // rows 128..255: the second pair of A boxes, same B
+                            umma_bf16(d1, smem_desc_sw128(sa + kABytes / 2 + k16 * a_step, a_lbo, 1024u), b_desc, idesc, (kb | k16) != 0u);
                     }
                     umma_commit(smem_u32(&sh.empty[s]));       // stage reusable once these MMAs are done
                 }
                 if (!ok) break;
-                umma_commit(smem_u32(&sh.acc_full[acc]));      // accumulator complete
-                ++acc_it;
+                umma_commit(smem_u32(&sh.acc_full[slot0]));    // accumulator(s) complete
+                if (slot0) ++used1; else ++used0;
+                if (tall) { umma_commit(smem_u32(&sh.acc_full[1])); ++used1; }
             }
             // drain: every MMA issued above has completed before tensor memory is released
             umma_commit(smem_u32(&sh.drain));
@@ -322,25 +338,37 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
                 if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(status, STATUS_TIMEOUT); break; }
         }
     } else if (warp >= kEpiWarp0) {
-        // ---- epilogue: accumulator -> registers -> packed partial block ----------------------------
+        // ---- epilogue: accumulator slot -> registers -> packed partial block --------------------------
+        const uint32_t group = (warp - kEpiWarp0) / kEpiWarpsPerGroup;   // the slot this warp drains
         const uint32_t quad = warp & 3u;                     // the 32 TMEM lanes this warp may read
         const uint32_t row = quad * 32u + lane;
-        uint32_t acc_it = 0;
+        uint32_t used = 0, toggle = 0;
         for (uint32_t i = 0;; ++i) {
             const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
             bool ok = mbar_wait(smem_u32(&sh.sched_full[q]), par, abort_flag, status);
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
             const uint32_t flags = sh.slot[q].flags, task = sh.slot[q].task, n_mma = sh.slot[q].n_mma;
-            const uint32_t rows = sh.slot[q].rows, cols = sh.slot[q].cols, ld = sh.slot[q].ld;
-            const uint64_t out_off = sh.slot[q].out_off;
+            const uint32_t tile_rows = sh.slot[q].rows, cols = sh.slot[q].cols, ld = sh.slot[q].ld;
+            uint64_t out_off = sh.slot[q].out_off;
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh.sched_empty[q]));
             if (flags & TILE_END) break;
-            const uint32_t acc = acc_it % kAccStages, aph = (acc_it / kAccStages) & 1u;
-            ok = mbar_wait(smem_u32(&sh.acc_full[acc]), aph, abort_flag, status);
+            // which half-tile, if any, lands in this group's slot (same rule as the MMA issuer)
+            uint32_t rows;
+            if (tile_rows > kBlockM) {
+                rows = group == 0 ? kBlockM : tile_rows - kBlockM;
+                out_off += (uint64_t)group * kBlockM * ld;
+            } else {
+                const bool mine = toggle == group;
+                toggle ^= 1u;
+                if (!mine) continue;
+                rows = tile_rows;
+            }
+            ok = mbar_wait(smem_u32(&sh.acc_full[group]), used & 1u, abort_flag, status);
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            ++used;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + acc * kAccCols + ((quad * 32u) << 16);
+            const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
             float* out_row = partials + out_off + (uint64_t)row * ld;
             const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
@@ -348,10 +376,10 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + c * 32u, v);
                 tmem_ld_wait();
-                if (c + 1 == nchunk) {                       // accumulator fully read: hand it back
+                if (c + 1 == nchunk) {                       // slot fully read: hand it back
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh.acc_empty[acc]));
+                    if (lane == 0) mbar_arrive(smem_u32(&sh.acc_empty[group]));
                 }
                 if (row < rows) {
                     const uint32_t c0 = c * 32u;
@@ -370,8 +398,7 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
             }
             __threadfence();
             __syncwarp();
-            if (lane == 0) atomicAdd(&done[task], 1u);       // bookkeeping: kEpiWarps counts per tile
-            ++acc_it;
+            if (lane == 0) atomicAdd(&done[task], 1u);       // bookkeeping: one count per warp and half-tile
         }
     }
 
@@ -393,7 +420,7 @@ __global__ void check_done_kernel(const cleave_task_t* tasks, const uint32_t* do
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_tasks) return;
     if (tasks[i].flags & CLEAVE_TASK_SUPERSEDED) return;
-    if (done[i] != ntiles[i] * kEpiWarps) atomicOr(status, STATUS_INCOMPLETE);
+    if (done[i] != ntiles[i] * kEpiWarpsPerGroup) atomicOr(status, STATUS_INCOMPLETE);
 }
 
 __global__ void collect_failed_kernel(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
@@ -401,7 +428,7 @@ __global__ void collect_failed_kernel(const cleave_task_t* tasks, const uint32_t
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_tasks) return;
     if (tasks[i].flags & CLEAVE_TASK_SUPERSEDED) return;
-    if (done[i] != ntiles[i] * kEpiWarps) out_ids[atomicAdd(out_count, 1u)] = i;
+    if (done[i] != ntiles[i] * kEpiWarpsPerGroup) out_ids[atomicAdd(out_count, 1u)] = i;
 }
 
 // -------------------------------------------------------------------------------------------------

@@ -10,23 +10,25 @@
 namespace cleave {
 
 // exec kernel geometry
-constexpr uint32_t kBlockM = 128;                    // MMA M: rows of a tile
+constexpr uint32_t kBlockM = 128;                    // MMA M: rows of a half-tile
+constexpr uint32_t kTileRows = 256;                  // rows of a tile: two halves sharing the B stage
 constexpr uint32_t kBlockNMax = 256;                 // widest MMA N
 constexpr uint32_t kBlockK = 64;                     // K per pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kSubRows = 64;                    // rows (or M/N elements) per TMA box
 constexpr uint32_t kSubBytes = kSubRows * kBlockK * 2;          // 8192: one 64 x 64 bf16 box
-constexpr uint32_t kABytes = 2 * kSubBytes;          // 128 rows of A
+constexpr uint32_t kABytes = 4 * kSubBytes;          // up to 256 rows of A
 constexpr uint32_t kBBytes = 4 * kSubBytes;          // up to 256 columns of B
-constexpr uint32_t kStageBytes = kABytes + kBBytes;  // 49152
-constexpr int kStages = 4;
-constexpr int kAccStages = 2;                        // accumulators in tensor memory (double buffer)
+constexpr uint32_t kStageBytes = kABytes + kBBytes;  // 65536
+constexpr int kStages = 3;
+constexpr int kAccSlots = 2;                         // accumulator slots in tensor memory
 constexpr uint32_t kAccCols = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSchedSlots = 4;
 constexpr uint32_t kExecDynSmem = kStages * kStageBytes + 1024;
 
-constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4, kEpiWarps = 4;
-constexpr int kExecThreads = 256;
+constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4;
+constexpr int kEpiWarpsPerGroup = 4, kEpiWarps = 2 * kEpiWarpsPerGroup;   // group g drains accumulator slot g
+constexpr int kExecThreads = 32 * (kEpiWarp0 + kEpiWarps);
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // bound of every device-side wait
 

@@ -9,7 +9,7 @@
 
 namespace cleave {
 
-// Work unit of the exec kernel: one (<=128 row) x (<=256 column) output tile of one task over the
+// Work unit of the exec kernel: one (<=256 row) x (<=256 column) output tile of one task over the
 // task's whole K-range.  64 bytes, read by the kernel's scheduler warp with four 16-byte loads.
 struct TileDesc {
     uint32_t task;      // owning task (bookkeeping)
@@ -19,7 +19,7 @@ struct TileDesc {
     uint32_t m_row;     // first row of the tile in op(A)
     uint32_t n_col;     // first column of the tile in op(B)
     uint32_t k0, k1;
-    uint32_t rows;      // valid rows   (1..128)
+    uint32_t rows;      // valid rows   (1..256)
     uint32_t cols;      // valid columns (1..256)
     uint32_t ld;        // leading dimension of the task's packed block (= beta)
     uint32_t pad0;

@@ -444,8 +444,8 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
 }
 
 // ---- exec work list -----------------------------------------------------------------------------
-// A task is cut into tiles of 128 rows x w columns, w <= 256 chosen so the column tiles are balanced
-// and 16-aligned.  Tiles are ordered so that tiles running at the same time share operand panels in
+// A task is cut into tiles of 256 rows x w columns, w <= 256 chosen so the column tiles are balanced
+// and 16-aligned (the kernel runs a tile as two 128-row halves that share the B operand).  Tiles are ordered so that tiles running at the same time share operand panels in
 // L2: by GEMM, K-range, band of 2048 rows, then column, then row.
 void build_tiles(cleave_plan_s& p, uint32_t first_task) {
     const uint32_t kBandRows = 2048;
@@ -460,22 +460,22 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
             p.exec_unsupported = 1;
         const uint32_t nt0 = (uint32_t)cdiv(beta, 256);
         const uint32_t w = (uint32_t)(cdiv(cdiv(beta, nt0), 16) * 16);
-        const uint32_t nt = (uint32_t)cdiv(beta, w), mt = (uint32_t)cdiv(alpha, 128);
-        p.task_ntiles[id] = nt * mt;
+        const uint32_t nt = (uint32_t)cdiv(beta, w), mt = (uint32_t)cdiv(alpha, 256);
+        p.task_ntiles[id] = nt * (uint32_t)cdiv(alpha, 128);      // bookkeeping counts 128-row half-tiles
         for (uint32_t ti = 0; ti < mt; ++ti)
             for (uint32_t tj = 0; tj < nt; ++tj) {
                 TileDesc d;
                 std::memset(&d, 0, sizeof d);
                 d.task = id; d.gemm = t.gemm;
                 d.flags = TILE_VALID | (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN);
-                d.rows = std::min(128u, alpha - ti * 128);
+                d.rows = std::min(256u, alpha - ti * 256);
                 d.cols = std::min(w, beta - tj * w);
                 d.n_mma = (d.cols + 15) / 16 * 16;
-                d.m_row = t.m0 + ti * 128;
+                d.m_row = t.m0 + ti * 256;
                 d.n_col = t.n0 + tj * w;
                 d.k0 = t.k0; d.k1 = t.k1;
                 d.ld = beta;
-                d.out_off = t.part_off + (uint64_t)ti * 128 * beta + (uint64_t)tj * w;
+                d.out_off = t.part_off + (uint64_t)ti * 256 * beta + (uint64_t)tj * w;
                 p.tiles.push_back(d);
             }
     }
