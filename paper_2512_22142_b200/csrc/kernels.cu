@@ -341,7 +341,8 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
         // ---- epilogue: accumulator slot -> registers -> packed partial block --------------------------
         const uint32_t group = (warp - kEpiWarp0) / kEpiWarpsPerGroup;   // the slot this warp drains
         const uint32_t quad = warp & 3u;                     // the 32 TMEM lanes this warp may read
-        const uint32_t row = quad * 32u + lane;
+        float* stage_tile = reinterpret_cast<float*>(dyn_smem + (stage_base - smem_u32(dyn_smem)) + kStages * kStageBytes) +
+                            (warp - kEpiWarp0) * kEpiStageFloats;
         uint32_t used = 0, toggle = 0;
         for (uint32_t i = 0;; ++i) {
             const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
@@ -369,8 +370,11 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
             ++used;
             tc_fence_after();
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
-            float* out_row = partials + out_off + (uint64_t)row * ld;
-            const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
+            // Thread `lane` holds row quad*32+lane of a 32-column chunk.  Stored from there, a warp store
+            // would touch 32 lines with 16 bytes each; the chunk is transposed through a padded 32 x 33
+            // staging tile instead, so that every warp store writes 128 contiguous bytes of one row.
+            float* out_blk = partials + out_off + (uint64_t)(quad * 32u) * ld;
+            const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
             const uint32_t nchunk = (n_mma + 31u) / 32u;
             for (uint32_t c = 0; c < nchunk; ++c) {
                 uint32_t v[32];
@@ -381,20 +385,16 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh.acc_empty[group]));
                 }
-                if (row < rows) {
-                    const uint32_t c0 = c * 32u;
-                    if (vec_ok && c0 + 32u <= cols) {
-                        float4* dst = reinterpret_cast<float4*>(out_row + c0);
 #pragma unroll
-                        for (int x = 0; x < 8; ++x)
-                            __stcs(dst + x, make_float4(__uint_as_float(v[4 * x]), __uint_as_float(v[4 * x + 1]),
-                                                        __uint_as_float(v[4 * x + 2]), __uint_as_float(v[4 * x + 3])));
-                    } else {
-#pragma unroll
-                        for (int x = 0; x < 32; ++x)
-                            if (c0 + x < cols) out_row[c0 + x] = __uint_as_float(v[x]);
-                    }
+                for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
+                __syncwarp();
+                const uint32_t col = c * 32u + lane;
+                if (col < cols) {
+                    float* dst = out_blk + col;
+#pragma unroll 8
+                    for (uint32_t r = 0; r < rows_here; ++r) __stcs(dst + (uint64_t)r * ld, stage_tile[r * 33 + lane]);
                 }
+                __syncwarp();
             }
             __threadfence();
             __syncwarp();

@@ -24,7 +24,8 @@ constexpr int kAccSlots = 2;                         // accumulator slots in ten
 constexpr uint32_t kAccCols = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSchedSlots = 4;
-constexpr uint32_t kExecDynSmem = kStages * kStageBytes + 1024;
+constexpr uint32_t kEpiStageFloats = 32 * 33;        // per epilogue warp: padded 32 x 32 transpose tile
+constexpr uint32_t kExecDynSmem = kStages * kStageBytes + 1024 + 8 * kEpiStageFloats * 4;
 
 constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4;
 constexpr int kEpiWarpsPerGroup = 4, kEpiWarps = 2 * kEpiWarpsPerGroup;   // group g drains accumulator slot g
