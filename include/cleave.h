@@ -86,7 +86,7 @@ typedef struct {
 
 /* Planner options.  Zero-initialise and call cleave_plan_opts_default. */
 typedef struct {
-    uint32_t gran_m, gran_n, gran_k;  /* block granularity in rows / columns / K (default 128)   */
+    uint32_t gran_m, gran_n, gran_k;  /* block granularity in rows / columns / K (256, 128, 128) */
     uint32_t kslice_max;              /* deepest K-slice, 0 = never split for depth (default 4096)*/
     uint32_t ksplit;                  /* 0 = automatic, else the forced number of K-slices        */
     uint32_t ksplit_cap;              /* upper limit of the automatic choice (default 8)          */

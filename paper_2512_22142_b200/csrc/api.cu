@@ -221,7 +221,8 @@ extern "C" {
 
 void cleave_plan_opts_default(cleave_plan_opts_t* o) {
     if (!o) return;
-    o->gran_m = o->gran_n = o->gran_k = 128;
+    o->gran_m = 256;            // rows of an exec-kernel tile: blocks of whole tiles waste no MMA work
+    o->gran_n = o->gran_k = 128;
     o->kslice_max = 4096;
     o->ksplit = 0;
     o->ksplit_cap = 8;

@@ -375,6 +375,7 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
             // staging tile instead, so that every warp store writes 128 contiguous bytes of one row.
             float* out_blk = partials + out_off + (uint64_t)(quad * 32u) * ld;
             const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
+            const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
             for (uint32_t c = 0; c < nchunk; ++c) {
                 uint32_t v[32];
@@ -388,11 +389,22 @@ exec_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int*
 #pragma unroll
                 for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
                 __syncwarp();
-                const uint32_t col = c * 32u + lane;
-                if (col < cols) {
-                    float* dst = out_blk + col;
+                const uint32_t c0 = c * 32u;
+                if (vec_ok && c0 + 32u <= cols) {
+                    // lane l: columns 4*(l%8) .. +3 of rows l/8, l/8+4, ...: one instruction writes 4 full rows
+                    const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
+                    float* dst = out_blk + c0 + cc;
+#pragma unroll
+                    for (uint32_t r = rr; r < 32u; r += 4u) {
+                        if (r < rows_here) {
+                            const float* src = stage_tile + r * 33 + cc;
+                            *reinterpret_cast<float4*>(dst + (uint64_t)r * ld) = make_float4(src[0], src[1], src[2], src[3]);
+                        }
+                    }
+                } else if (c0 + lane < cols) {
+                    float* dst = out_blk + c0 + lane;
 #pragma unroll 8
-                    for (uint32_t r = 0; r < rows_here; ++r) __stcs(dst + (uint64_t)r * ld, stage_tile[r * 33 + lane]);
+                    for (uint32_t r = 0; r < rows_here; ++r) dst[(uint64_t)r * ld] = stage_tile[r * 33 + lane];
                 }
                 __syncwarp();
             }
