@@ -45,6 +45,7 @@ extern "C" {
 #define CLEAVE_E_BOUNDS       -8   /* a device-side range check failed; the access was skipped     */
 #define CLEAVE_E_INCOMPLETE   -9   /* assembly read a block whose task never finished              */
 #define CLEAVE_E_NOMEM        -10  /* host or device allocation failed                             */
+#define CLEAVE_E_TOOBIG       -11  /* the plan's tables exceed CLEAVE_STATIC_SCRATCH_BYTES         */
 
 /* ---- records ----------------------------------------------------------------------------- */
 
@@ -186,6 +187,34 @@ CLEAVE_API uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task)
 /* Device time of the last exec-kernel and assembly-kernel launches on this plan, in
  * milliseconds, measured with CUDA events on the launching stream (synchronises those events). */
 CLEAVE_API int cleave_last_kernel_ms(cleave_plan_t* p, float* exec_ms, float* assemble_ms);
+
+/* cleave_assemble for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this is a convenience of the library.)
+ *
+ * Some hosts of this library hand all device memory to a pool of their own (a serving process
+ * that sizes its caches to the last byte, a framework allocator with a hard memory fraction): a
+ * cudaMalloc made behind their back fails or defeats their accounting.  Others sit in a
+ * latency-critical loop where cudaMalloc / cudaFree would stall every stream of the device.
+ * cleave_assemble allocates its lookup tables on a plan's first use; this variant never calls
+ * cudaMalloc, cudaFree or any allocating routine.  Its tables live in a fixed array of
+ * CLEAVE_STATIC_SCRATCH_BYTES that belongs to the library image: every device that loads the
+ * library holds that much memory until the process exits.
+ *
+ *   - Same inputs, outputs and arithmetic as cleave_assemble (bit-identical sums); the caller owns
+ *     partials and every C[i].  It performs no bookkeeping check: E_INCOMPLETE is never raised, so
+ *     use it after a cleave_exec / cleave_reissue that is known to have run every task.
+ *   - A plan whose tables do not fit the array is refused with CLEAVE_E_TOOBIG before anything is
+ *     launched (about 50 bytes per 16K outputs: the Llama-7B-shaped layer needs ~3 MiB and is
+ *     refused, a layer of a quarter of that size fits).
+ *   - The first call on each device asks the runtime for the array's address on that device (with
+ *     that device current).  Make this first call outside any stream capture.
+ *   - All calls share the one array, and it keeps what the last call wrote.  Each call rewrites
+ *     every byte its kernels read, in stream order; two calls whose work overlaps on the GPU (on
+ *     different streams, or from different threads) race on the array and must be serialised by the
+ *     caller.
+ * Errors: E_INVAL, E_UNSUPPORTED (more than 32 K-slices), E_TOOBIG, E_CUDA. */
+#define CLEAVE_STATIC_SCRATCH_BYTES (2u << 20)
+CLEAVE_API int cleave_assemble_static(cleave_plan_t* p, const float* partials, float* const* C, void* stream);
 
 CLEAVE_API void cleave_destroy(cleave_plan_t* p);
 CLEAVE_API const char* cleave_strerror(int code);

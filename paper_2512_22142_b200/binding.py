@@ -49,6 +49,7 @@ _sig = {
     "cleave_set_drops": (_i, [_vp, _vp, _u32]),
     "cleave_exec": (_i, [_vp, _vp, _vp, _vp, _vp]),
     "cleave_assemble": (_i, [_vp, _vp, _vp, _vp]),
+    "cleave_assemble_static": (_i, [_vp, _vp, _vp, _vp]),
     "cleave_reissue": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp]),
     "cleave_replan": (_i, [_vp, _vp, _u32, C.POINTER(_u32)]),
     "cleave_status": (_i, [_vp, _vp]),
@@ -180,6 +181,13 @@ class Plan:
     def assemble(self, partials, Cs, stream=None) -> None:
         pc = _ptr_array(Cs)
         _check(lib.cleave_assemble(self._h, partials.data_ptr(), pc.ctypes.data, _stream(stream)), "cleave_assemble")
+
+    def assemble_static(self, partials, Cs, stream=None) -> None:
+        """cleave_assemble_static: the assembly for callers that must not allocate device memory (its
+        tables live in a fixed array inside the library; plans too large for it raise E_TOOBIG)."""
+        pc = _ptr_array(Cs)
+        _check(lib.cleave_assemble_static(self._h, partials if isinstance(partials, int) else partials.data_ptr(),
+                                          pc.ctypes.data, _stream(stream)), "cleave_assemble_static")
 
     def reissue(self, failed, A, B, partials, stream=None) -> None:
         f = np.ascontiguousarray(failed if failed is not None else [], dtype=np.uint32)

@@ -414,6 +414,7 @@ const char* cleave_strerror(int code) {
         case CLEAVE_E_BOUNDS: return "device-side range check failed";
         case CLEAVE_E_INCOMPLETE: return "a task feeding the assembly never finished";
         case CLEAVE_E_NOMEM: return "out of memory";
+        case CLEAVE_E_TOOBIG: return "plan tables exceed the fixed scratch array (CLEAVE_STATIC_SCRATCH_BYTES)";
         default: return "unknown error";
     }
 }

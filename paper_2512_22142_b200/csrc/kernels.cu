@@ -18,6 +18,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "cleave.h"
 #include "kernels.cuh"
 
 namespace cleave {
@@ -599,3 +600,69 @@ cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t i
 }
 
 }  // namespace cleave
+
+// -------------------------------------------------------------------------------------------------
+// cleave_assemble_static: assembly without any allocation
+// -------------------------------------------------------------------------------------------------
+// The assembly kernels read three small tables from device memory (work items, block references,
+// output pointers and leading dimensions).  cleave_assemble keeps them in buffers it allocates on
+// the plan's first use.  This entry point is for callers that must not allocate: it keeps the
+// tables in one fixed array that is part of the loaded library image, so no cudaMalloc / cudaFree
+// happens here, ever.  Every device that loads the library holds CLEAVE_STATIC_SCRATCH_BYTES for it
+// until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[CLEAVE_STATIC_SCRATCH_BYTES];
+
+namespace {
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address: the
+// address on the current device has to be asked for, once per device.
+unsigned char* static_scratch_on_current_device(int* rc) {
+    static unsigned char* cached[64] = {nullptr};
+    int dev = -1;
+    *rc = CLEAVE_E_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return nullptr; }
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return nullptr; }
+        cached[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *rc = 0;
+    return cached[dev];
+}
+inline size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+}  // namespace
+
+extern "C" int cleave_assemble_static(cleave_plan_t* p, const float* partials, float* const* C, void* stream) {
+    if (!p || !partials || !C) return CLEAVE_E_INVAL;
+    for (uint32_t s : p->ksplit) if (s > 32) return CLEAVE_E_UNSUPPORTED;
+    const size_t n = p->gemms.size();
+    for (size_t i = 0; i < n; ++i) if (!C[i] || ((uintptr_t)C[i] & 15)) return CLEAVE_E_INVAL;
+    // layout of the fixed array: items | refs | output pointers | leading dimensions
+    const size_t items_b = p->asm_items.size() * sizeof(cleave::AsmItem), refs_b = p->asm_refs.size() * sizeof(cleave::AsmRef);
+    const size_t off_refs = round256(items_b), off_ptrs = off_refs + round256(refs_b), off_ld = off_ptrs + round256(n * sizeof(float*));
+    if (off_ld + n * sizeof(uint32_t) > (size_t)CLEAVE_STATIC_SCRATCH_BYTES) return CLEAVE_E_TOOBIG;
+    int rc = 0;
+    unsigned char* base = static_scratch_on_current_device(&rc);
+    if (!base) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t ldc[1024];
+    if (n > 1024) return CLEAVE_E_TOOBIG;
+    for (size_t i = 0; i < n; ++i) ldc[i] = p->gemms[i].N;
+    // Everything the kernels read is rewritten by these copies, so nothing left by an earlier call is used.
+    if (cudaMemcpyAsync(base, p->asm_items.data(), items_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(base + off_refs, p->asm_refs.data(), refs_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(base + off_ptrs, C, n * sizeof(float*), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(base + off_ld, ldc, n * sizeof(uint32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return CLEAVE_E_CUDA;
+    }
+    for (const auto& grp : p->asm_groups) {
+        if (cleave::launch_assemble(reinterpret_cast<const cleave::AsmItem*>(base), reinterpret_cast<const cleave::AsmRef*>(base + off_refs),
+                                    grp.item0, grp.n_items, grp.sp, partials, reinterpret_cast<float* const*>(base + off_ptrs),
+                                    reinterpret_cast<const uint32_t*>(base + off_ld), st) != cudaSuccess) {
+            cudaGetLastError();
+            return CLEAVE_E_CUDA;
+        }
+    }
+    return 0;
+}
+
