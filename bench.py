@@ -201,6 +201,24 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------------
+# rank plumbing (replicas only: no collective on the data path)
+# --------------------------------------------------------------------------------------------------
+def rank_max(x: float, dist, device) -> float:
+    """The slowest rank's time: every rank reports the same number."""
+    if dist is None:
+        return x
+    import torch
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(flop_per_replica: float, world: int, ms_per_step: float) -> float:
+    """Whole-job TFLOP/s of `world` independent replicas that all finish a step in ms_per_step."""
+    return world * flop_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
+# --------------------------------------------------------------------------------------------------
 # the CUDA path
 # --------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -249,11 +267,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return rank_max(x, dist, dev)
 
     # ---- device-resident steps -------------------------------------------------------------------
     for _ in range(args.warmup):
@@ -281,7 +295,7 @@ def run_ours(args):
     exec_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     asm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
     ms_per_step = total_ms / args.steps
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value = job_throughput(flops, world, ms_per_step)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----------------
     host_C = [torch.empty((g.M, g.N), dtype=torch.float32).pin_memory() if args.e2e_steps > 0 else
@@ -307,7 +321,7 @@ def run_ours(args):
     e2.record()
     barrier()
     e2e_ms = max_over_ranks(b2.elapsed_time(e2)) / max(args.e2e_steps, 1) if args.e2e_steps > 0 else float("nan")
-    e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
+    e2e_value = job_throughput(flops, world, e2e_ms)
     checksum = float(host_C[0][0, :8].double().sum())
 
     if rank != 0:
