@@ -10,8 +10,8 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB_DIR = os.path.join(PKG, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libcleave.so")
-SOURCES = ["planner.cpp", "kernels.cu", "api.cu"]
-HEADERS = ["plan_internal.hpp", "kernels.cuh", os.path.join(ROOT, "include", "cleave.h")]
+SOURCES = ["planner.cpp", "kernels.cu", "kernels_pair.cu", "api.cu"]
+HEADERS = ["plan_internal.hpp", "kernels.cuh", "ptx.cuh", os.path.join(ROOT, "include", "cleave.h")]
 
 
 def _nvcc() -> str:

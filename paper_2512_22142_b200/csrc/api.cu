@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -92,6 +93,7 @@ int sync_device_state(cleave_plan_s* p, cudaStream_t st) {
         CU_TRY(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, d->device));
         if (cc_major != 10) return CLEAVE_E_UNSUPPORTED;
         CU_TRY(exec_kernel_prepare());
+        CU_TRY(exec_pair_kernel_prepare());
         RC_TRY(dev_alloc(&d->words, 4));
         CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
         RC_TRY(dev_alloc(&d->maps, 2 * p->gemms.size()));
@@ -187,6 +189,10 @@ int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, uint32_t
     if (tile_end > tile_begin) {
         const uint32_t grid = std::min<uint32_t>((uint32_t)d->sm_count, tile_end - tile_begin);
         CU_TRY(cudaEventRecord(d->ev[0], st));
+        if (getenv("CLEAVE_EXEC_PAIR")) {
+            const uint32_t clusters = std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)d->sm_count / 2, tile_end - tile_begin));
+            CU_TRY(launch_exec_pair(clusters, d->tiles, tile_end, d->words + 0, d->maps, partials, d->done, d->words + 1, st));
+        } else
         CU_TRY(launch_exec(grid, d->tiles, tile_end, d->words + 0, d->maps, partials, d->done, d->words + 1, st));
         CU_TRY(cudaEventRecord(d->ev[1], st));
         d->ev_exec = true;

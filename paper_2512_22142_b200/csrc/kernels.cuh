@@ -27,6 +27,13 @@ constexpr int kSchedSlots = 4;
 constexpr uint32_t kEpiStageFloats = 32 * 33;        // per epilogue warp: padded 32 x 32 transpose tile
 constexpr uint32_t kExecDynSmem = kStages * kStageBytes + 1024 + 8 * kEpiStageFloats * 4;
 
+// pair kernel (two CTAs per tile): per CTA 128 rows of A and half of the columns of B per stage
+constexpr uint32_t kPairABytes = 2 * kSubBytes;
+constexpr uint32_t kPairBBytes = 2 * kSubBytes;
+constexpr uint32_t kPairStageBytes = kPairABytes + kPairBBytes;   // 32768
+constexpr int kPairStages = 6;
+constexpr uint32_t kPairDynSmem = kPairStages * kPairStageBytes + 1024 + 8 * kEpiStageFloats * 4;
+
 constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4;
 constexpr int kEpiWarpsPerGroup = 4, kEpiWarps = 2 * kEpiWarpsPerGroup;   // group g drains accumulator slot g
 constexpr int kExecThreads = 32 * (kEpiWarp0 + kEpiWarps);
@@ -42,6 +49,9 @@ cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile
 cudaError_t exec_kernel_prepare();
 cudaError_t launch_exec(uint32_t grid, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
                         const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status, cudaStream_t st);
+cudaError_t exec_pair_kernel_prepare();
+cudaError_t launch_exec_pair(uint32_t clusters, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
+                             const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status, cudaStream_t st);
 cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles, uint32_t n_tasks,
                               unsigned int* status, cudaStream_t st);
 cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
