@@ -259,7 +259,8 @@ def run_ours(args):
     C = [torch.empty((g.M, g.N), dtype=torch.float32, device=dev) for g in w.gemms]
     flops = float(w.flops)
     S = [plan.ksplit(i) for i in range(len(w.gemms))]
-    asm_bytes = float(sum((S[i] + 1) * g.M * g.N * 4 for i, g in enumerate(w.gemms)))
+    # bytes the assembly kernels move: GEMMs with one K-slice are finished by the exec kernel in fused mode
+    asm_bytes = float(sum((S[i] + 1) * g.M * g.N * 4 for i, g in enumerate(w.gemms) if args.two_step or S[i] > 1))
 
     def barrier():
         if dist is not None:
@@ -270,8 +271,15 @@ def run_ours(args):
         return rank_max(x, dist, dev)
 
     # ---- device-resident steps -------------------------------------------------------------------
+    def run_exec():
+        # one-slice GEMMs are written straight to C by the exec kernel unless --two-step is given
+        if args.two_step:
+            plan.exec(A, B, partials)
+        else:
+            plan.exec_fused(A, B, partials, C)
+
     for _ in range(args.warmup):
-        plan.exec(A, B, partials)
+        run_exec()
         plan.assemble(partials, C)
     plan.check_status()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
@@ -283,7 +291,7 @@ def run_ours(args):
     begin.record()
     for s in range(args.steps):
         ev[s][0].record()
-        plan.exec(A, B, partials)
+        run_exec()
         ev[s][1].record()
         plan.assemble(partials, C)
         ev[s][2].record()
@@ -306,7 +314,7 @@ def run_ours(args):
     def e2e_step():
         for k, t in tensors.items():
             d_tensors[k].copy_(t, non_blocking=True)
-        plan.exec(A, B, partials)
+        run_exec()
         plan.assemble(partials, C)
         for hc, c in zip(host_C, C):
             hc.copy_(c, non_blocking=True)
@@ -335,7 +343,10 @@ def run_ours(args):
         p2 = cl.plan(w.gemms, devs, cl.default_opts(**opts))
         failed = ci.make_failed_ids(p2.num_tasks, 0.10, w.seed + 2)
         p2.set_drops(failed)
-        p2.exec(A, B, partials)
+        if args.two_step:
+            p2.exec(A, B, partials)
+        else:
+            p2.exec_fused(A, B, partials, C)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         c0, c1, c2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
@@ -362,6 +373,7 @@ def run_ours(args):
             "workload": w.name, "gemms": len(w.gemms), "devices": w.n_devices, "tasks": plan.num_tasks,
             "tiles": plan.num_tiles, "flop_per_step": flops, "ksplit": S, "arena_GB": plan.arena_elems * 4 / 1e9,
             "parallelism": "replicas only" if world > 1 else "1 GPU",
+            "write_out": "two-step" if args.two_step else "fused for one-slice GEMMs",
             "l2": "not flushed; operands + arena + outputs per step (~%.1f GB) far exceed the 126 MB L2" %
                   ((h2d + plan.arena_elems * 4 + d2h) / 1e9),
             "plan_ms_host": plan_ms, "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
@@ -369,7 +381,7 @@ def run_ours(args):
             "pct_of_measured_sustained_bf16": 100 * value / world / peaks["bf16_tflops_sustained"],
             "churn": churn, "e2e_ms_per_step": e2e_ms, "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
         },
-        "roofline": {"kernel": "exec_kernel", "bound": "tensor", "achieved": exec_tflops, "peak": peaks["bf16_tflops_sustained"],
+        "roofline": {"kernel": "exec_pair_kernel", "bound": "tensor", "achieved": exec_tflops, "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": exec_tflops / peaks["bf16_tflops_sustained"], "traffic": None,
                      "peak_kind": f"{peak_kind}, sustained cuBLAS bf16 (kernel timed inside a long step)",
                      "frac_of_burst": exec_tflops / peaks["bf16_tflops"], "frac_of_nominal": exec_tflops / NOMINAL_BF16_TFLOPS},
@@ -400,6 +412,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-churn", action="store_true")
+    ap.add_argument("--two-step", action="store_true", help="cleave_exec + full cleave_assemble instead of the fused write-out")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -127,7 +127,7 @@ CLEAVE_API uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gem
 CLEAVE_API uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm);     /* water-fill level    */
 CLEAVE_API uint32_t cleave_plan_num_tiles(const cleave_plan_t* p);        /* work units of the exec kernel  */
 CLEAVE_API uint32_t cleave_plan_num_launches(const cleave_plan_t* p);     /* kernels launched by one
-                                                  cleave_exec followed by one cleave_assemble    */
+                                   cleave_exec[_fused] + cleave_assemble, in the current mode    */
 
 /* Host-made failures (Section 3.2, "Device departures are detected via disconnect events"): the
  * listed tasks are skipped by every later cleave_exec / cleave_reissue launch, as if their device
@@ -147,6 +147,19 @@ CLEAVE_API int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t 
  * Errors: E_INVAL, E_UNSUPPORTED, E_CUDA, E_NOMEM. */
 CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
                 void* stream);
+
+/* cleave_exec with the write-out of one-slice GEMMs fused into the sub-GEMM kernel.  For a GEMM
+ * with a single K-slice a device's block is already a finished block of O (Section 4.1, "each
+ * device computes A' o B', a subset of O_s"; the paper's own formulation), so the kernel stores it
+ * at its place in C_g instead of the arena and the following cleave_assemble has nothing to do for
+ * that GEMM; GEMMs with several K-slices go through the arena as in cleave_exec.  The results are
+ * bit-identical to cleave_exec + cleave_assemble.
+ *   C [host array of n_gemms device pointers, fp32 row-major, ld = N, 16-byte aligned].  The same C
+ *   must be passed to the cleave_assemble that follows; cleave_reissue after a fused execution writes
+ *   replacement blocks of one-slice GEMMs to that C as well.  A plain cleave_exec ends fused mode.
+ * Errors: as cleave_exec. */
+CLEAVE_API int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
+                                 float* const* C, void* stream);
 
 /* Parameter-server aggregation (Section 3.1 / 3.2: the server "aggregates the computed outputs";
  * with a K-split it is a sum): C_g[i,j] = sum over the K-slices s of the partial block covering

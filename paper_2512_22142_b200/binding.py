@@ -48,6 +48,7 @@ _sig = {
     "cleave_plan_num_launches": (_u32, [_vp]),
     "cleave_set_drops": (_i, [_vp, _vp, _u32]),
     "cleave_exec": (_i, [_vp, _vp, _vp, _vp, _vp]),
+    "cleave_exec_fused": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "cleave_assemble": (_i, [_vp, _vp, _vp, _vp]),
     "cleave_assemble_static": (_i, [_vp, _vp, _vp, _vp]),
     "cleave_reissue": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp]),
@@ -177,6 +178,11 @@ class Plan:
         pa, pb = _ptr_array(A), _ptr_array(B)
         _check(lib.cleave_exec(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(), _stream(stream)),
                "cleave_exec")
+
+    def exec_fused(self, A, B, partials, Cs, stream=None) -> None:
+        pa, pb, pc = _ptr_array(A), _ptr_array(B), _ptr_array(Cs)
+        _check(lib.cleave_exec_fused(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(), pc.ctypes.data,
+                                     _stream(stream)), "cleave_exec_fused")
 
     def assemble(self, partials, Cs, stream=None) -> None:
         pc = _ptr_array(Cs)

@@ -4,7 +4,6 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -92,7 +91,6 @@ int sync_device_state(cleave_plan_s* p, cudaStream_t st) {
         int cc_major = 0;
         CU_TRY(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, d->device));
         if (cc_major != 10) return CLEAVE_E_UNSUPPORTED;
-        CU_TRY(exec_kernel_prepare());
         CU_TRY(exec_pair_kernel_prepare());
         RC_TRY(dev_alloc(&d->words, 4));
         CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
@@ -181,19 +179,27 @@ int check_exec_args(cleave_plan_s* p, const void* const* A, const void* const* B
     return 0;
 }
 
+int upload_c_ptrs(cleave_plan_s* p, float* const* C, cudaStream_t st) {
+    DeviceState* d = p->dev;
+    const size_t n = p->gemms.size();
+    for (size_t i = 0; i < n; ++i) if (!C[i] || ((uintptr_t)C[i] & 15)) return CLEAVE_E_INVAL;
+    if (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin())) {
+        d->last_c.assign(C, C + n);
+        CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(float*), cudaMemcpyHostToDevice, st));
+    }
+    return 0;
+}
+
 int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, uint32_t task_begin, uint32_t task_end,
               int clear_status, float* partials, cudaStream_t st) {
     DeviceState* d = p->dev;
     CU_TRY(launch_arm_queue(d->tiles, tile_begin, tile_end, d->tasks, d->dropped, d->done, task_begin, task_end,
-                            d->words + 0, d->words + 1, clear_status, st));
+                            d->words + 0, d->words + 1, clear_status, p->fused ? 1 : 0, st));
     if (tile_end > tile_begin) {
-        const uint32_t grid = std::min<uint32_t>((uint32_t)d->sm_count, tile_end - tile_begin);
+        // one cluster of two CTAs per pair of SMs, never more clusters than tiles
+        const uint32_t clusters = std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)d->sm_count / 2, tile_end - tile_begin));
         CU_TRY(cudaEventRecord(d->ev[0], st));
-        if (getenv("CLEAVE_EXEC_PAIR")) {
-            const uint32_t clusters = std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)d->sm_count / 2, tile_end - tile_begin));
-            CU_TRY(launch_exec_pair(clusters, d->tiles, tile_end, d->words + 0, d->maps, partials, d->done, d->words + 1, st));
-        } else
-        CU_TRY(launch_exec(grid, d->tiles, tile_end, d->words + 0, d->maps, partials, d->done, d->words + 1, st));
+        CU_TRY(launch_exec_pair(clusters, d->tiles, tile_end, d->words + 0, d->maps, partials, d->c_ptrs, d->done, d->words + 1, st));
         CU_TRY(cudaEventRecord(d->ev[1], st));
         d->ev_exec = true;
     }
@@ -282,7 +288,12 @@ uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm) { return
 uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->tstar.size()) ? p->tstar[gemm] : 0; }
 uint32_t cleave_plan_num_tiles(const cleave_plan_t* p) { return p ? (uint32_t)p->tiles.size() : 0; }
 // exec: arm + grouped GEMM; assemble: clear verdict + bookkeeping check + one kernel per slice-count class
-uint32_t cleave_plan_num_launches(const cleave_plan_t* p) { return p ? 4u + (uint32_t)p->asm_groups.size() : 0; }
+uint32_t cleave_plan_num_launches(const cleave_plan_t* p) {
+    if (!p) return 0;
+    uint32_t n = 4;
+    for (const auto& grp : p->asm_groups) if (!(p->fused && grp.single)) ++n;
+    return n;
+}
 uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task) { return (p && task < p->task_ntiles.size()) ? p->task_ntiles[task] : 0; }
 
 int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t n) {
@@ -302,6 +313,22 @@ int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, fl
         RC_TRY(sync_device_state(p, st));
         RC_TRY(update_maps(p, A, B, st));
     } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    p->fused = false;
+    return run_tiles(p, 0, (uint32_t)p->tiles.size(), 0, (uint32_t)p->tasks.size(), 1, partials, st);
+}
+
+int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials, float* const* C,
+                      void* stream) {
+    int rc = check_exec_args(p, A, B, partials);
+    if (rc) return rc;
+    if (!C) return CLEAVE_E_INVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    try {
+        RC_TRY(sync_device_state(p, st));
+        RC_TRY(update_maps(p, A, B, st));
+        RC_TRY(upload_c_ptrs(p, C, st));
+    } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    p->fused = true;
     return run_tiles(p, 0, (uint32_t)p->tiles.size(), 0, (uint32_t)p->tasks.size(), 1, partials, st);
 }
 
@@ -312,14 +339,13 @@ int cleave_assemble(cleave_plan_t* p, const float* partials, float* const* C, vo
     try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     DeviceState* d = p->dev;
     const size_t n = p->gemms.size();
-    for (size_t i = 0; i < n; ++i) if (!C[i] || ((uintptr_t)C[i] & 15)) return CLEAVE_E_INVAL;
-    if (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin())) {
-        d->last_c.assign(C, C + n);
-        CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(float*), cudaMemcpyHostToDevice, st));
-    }
+    // after a fused execution part of the result already sits in the C it was given: it must be the same C
+    if (p->fused && (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin()))) return CLEAVE_E_INVAL;
+    try { RC_TRY(upload_c_ptrs(p, C, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     CU_TRY(launch_check_done(d->tasks, d->done, d->ntiles, d->tasks_n, d->words + 1, st));
     CU_TRY(cudaEventRecord(d->ev[2], st));
     for (const auto& grp : p->asm_groups)
+        if (!(p->fused && grp.single))            // one-slice blocks were written to C by the exec kernel
         CU_TRY(launch_assemble(d->asm_items, d->asm_refs, grp.item0, grp.n_items, grp.sp, partials, d->c_ptrs, d->ldcs, st));
     CU_TRY(cudaEventRecord(d->ev[3], st));
     d->ev_asm = true;

@@ -9,34 +9,26 @@
 
 namespace cleave {
 
-// exec kernel geometry
-constexpr uint32_t kBlockM = 128;                    // MMA M: rows of a half-tile
-constexpr uint32_t kTileRows = 256;                  // rows of a tile: two halves sharing the B stage
+// exec kernel geometry: a tile of <= 256 rows x <= 256 columns is run by a pair of CTAs
+constexpr uint32_t kBlockM = 128;                    // rows of a tile owned by one CTA of the pair
 constexpr uint32_t kBlockNMax = 256;                 // widest MMA N
 constexpr uint32_t kBlockK = 64;                     // K per pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kSubRows = 64;                    // rows (or M/N elements) per TMA box
 constexpr uint32_t kSubBytes = kSubRows * kBlockK * 2;          // 8192: one 64 x 64 bf16 box
-constexpr uint32_t kABytes = 4 * kSubBytes;          // up to 256 rows of A
-constexpr uint32_t kBBytes = 4 * kSubBytes;          // up to 256 columns of B
-constexpr uint32_t kStageBytes = kABytes + kBBytes;  // 65536
-constexpr int kStages = 3;
-constexpr int kAccSlots = 2;                         // accumulator slots in tensor memory
+constexpr uint32_t kPairABytes = 2 * kSubBytes;      // per CTA and stage: 128 rows of A ...
+constexpr uint32_t kPairBBytes = 2 * kSubBytes;      // ... and half of the (<= 256) columns of B
+constexpr uint32_t kPairStageBytes = kPairABytes + kPairBBytes;   // 32768
+constexpr int kPairStages = 6;
+constexpr int kAccSlots = 2;                         // accumulator slots in tensor memory (double buffer)
 constexpr uint32_t kAccCols = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSchedSlots = 4;
 constexpr uint32_t kEpiStageFloats = 32 * 33;        // per epilogue warp: padded 32 x 32 transpose tile
-constexpr uint32_t kExecDynSmem = kStages * kStageBytes + 1024 + 8 * kEpiStageFloats * 4;
-
-// pair kernel (two CTAs per tile): per CTA 128 rows of A and half of the columns of B per stage
-constexpr uint32_t kPairABytes = 2 * kSubBytes;
-constexpr uint32_t kPairBBytes = 2 * kSubBytes;
-constexpr uint32_t kPairStageBytes = kPairABytes + kPairBBytes;   // 32768
-constexpr int kPairStages = 6;
-constexpr uint32_t kPairDynSmem = kPairStages * kPairStageBytes + 1024 + 8 * kEpiStageFloats * 4;
 
 constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4;
 constexpr int kEpiWarpsPerGroup = 4, kEpiWarps = 2 * kEpiWarpsPerGroup;   // group g drains accumulator slot g
 constexpr int kExecThreads = 32 * (kEpiWarp0 + kEpiWarps);
+constexpr uint32_t kPairDynSmem = kPairStages * kPairStageBytes + 1024 + kEpiWarps * kEpiStageFloats * 4;
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // bound of every device-side wait
 
@@ -45,13 +37,11 @@ enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BOUNDS = 2u, STATUS_INCOMPLETE
 
 cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
                              const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                             unsigned int* ticket, unsigned int* status, int clear_status, cudaStream_t st);
-cudaError_t exec_kernel_prepare();
-cudaError_t launch_exec(uint32_t grid, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
-                        const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status, cudaStream_t st);
+                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, cudaStream_t st);
 cudaError_t exec_pair_kernel_prepare();
 cudaError_t launch_exec_pair(uint32_t clusters, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
-                             const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status, cudaStream_t st);
+                             const CUtensorMap* maps, float* partials, float* const* c_ptrs, uint32_t* done,
+                             unsigned int* status, cudaStream_t st);
 cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles, uint32_t n_tasks,
                               unsigned int* status, cudaStream_t st);
 cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,

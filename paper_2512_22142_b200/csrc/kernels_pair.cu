@@ -17,7 +17,12 @@
 //   sched ring   the leader's scheduler warp pops the ticket, writes the tile descriptor into both
 //                CTAs' slot rings and arrives on both CTAs' sched_full; every consumer of either
 //                CTA arrives on the leader's sched_empty
-// No TMA load uses cluster multicast.  Every wait is bounded, as in exec_kernel.
+// No TMA load uses cluster multicast.
+//
+// Every device-side wait is bounded: when a wait expires the CTA records E_TIMEOUT in the status
+// word and raises its abort flag, all its roles leave their loops, the MMAs in flight are drained
+// (again with a bound), both CTAs meet at the cluster barrier, tensor memory is released and the
+// kernel returns.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -136,7 +141,8 @@ struct __align__(16) PairShared {
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kExecThreads, 1)
 exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int* ticket,
-                 const CUtensorMap* __restrict__ maps, float* __restrict__ partials, uint32_t* done, unsigned int* status) {
+                 const CUtensorMap* __restrict__ maps, float* __restrict__ partials, float* const* __restrict__ c_ptrs,
+                 uint32_t* done, unsigned int* status) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ PairShared sh;
 
@@ -285,8 +291,11 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
             bool ok = mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, abort_flag, status);
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
             const uint32_t flags = sh.slot[q].flags, task = sh.slot[q].task, n_mma = sh.slot[q].n_mma;
-            const uint32_t tile_rows = sh.slot[q].rows, cols = sh.slot[q].cols, ld = sh.slot[q].ld;
-            const uint64_t out_off = sh.slot[q].out_off + (uint64_t)rank * kBlockM * ld;
+            const uint32_t tile_rows = sh.slot[q].rows, cols = sh.slot[q].cols, gemm = sh.slot[q].gemm;
+            // a block of a one-slice GEMM is final: it may go straight to its place in C
+            const bool direct = flags & TILE_DIRECT;
+            const uint32_t ld = direct ? sh.slot[q].ldc : sh.slot[q].ld;
+            const uint64_t out_off = (direct ? sh.slot[q].c_off : sh.slot[q].out_off) + (uint64_t)rank * kBlockM * ld;
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
             if (flags & TILE_END) break;
@@ -299,7 +308,7 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
             ++used;
             tc_fence_after();
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
-            float* out_blk = partials + out_off + (uint64_t)(quad * 32u) * ld;
+            float* out_blk = (direct ? c_ptrs[gemm] : partials) + out_off + (uint64_t)(quad * 32u) * ld;
             const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
             const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
@@ -356,8 +365,9 @@ cudaError_t exec_pair_kernel_prepare() {
 }
 
 cudaError_t launch_exec_pair(uint32_t clusters, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
-                             const CUtensorMap* maps, float* partials, uint32_t* done, unsigned int* status, cudaStream_t st) {
-    exec_pair_kernel<<<2 * clusters, kExecThreads, kPairDynSmem, st>>>(tiles, tile_end, ticket, maps, partials, done, status);
+                             const CUtensorMap* maps, float* partials, float* const* c_ptrs, uint32_t* done,
+                             unsigned int* status, cudaStream_t st) {
+    exec_pair_kernel<<<2 * clusters, kExecThreads, kPairDynSmem, st>>>(tiles, tile_end, ticket, maps, partials, c_ptrs, done, status);
     return cudaGetLastError();
 }
 

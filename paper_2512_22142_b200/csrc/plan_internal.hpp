@@ -22,14 +22,16 @@ struct TileDesc {
     uint32_t rows;      // valid rows   (1..256)
     uint32_t cols;      // valid columns (1..256)
     uint32_t ld;        // leading dimension of the task's packed block (= beta)
-    uint32_t pad0;
+    uint32_t ldc;       // leading dimension of the GEMM's C (= N)
     uint64_t out_off;   // fp32 element offset of the tile's (0,0) in the arena
-    uint64_t pad1;
+    uint64_t c_off;     // element offset of the tile's (0,0) in C
 };
 static_assert(sizeof(TileDesc) == 64, "TileDesc must be 64 bytes");
 
 // A_MN / B_MN: the operand is stored with M (resp. N) contiguous (transA = 1, resp. transB = 0)
-enum : uint32_t { TILE_VALID = 1u, TILE_END = 2u, TILE_A_MN = 4u, TILE_B_MN = 8u };
+// SINGLE: the GEMM has one K-slice, so the tile's block is already the final value of C there;
+// DIRECT: (set per launch) write it to C instead of the arena
+enum : uint32_t { TILE_VALID = 1u, TILE_END = 2u, TILE_A_MN = 4u, TILE_B_MN = 8u, TILE_SINGLE = 16u, TILE_DIRECT = 32u };
 
 // One unit of assembly work: `nrows` full rows of a rectangle of C in which every K-slice is
 // served by one task.  `ref0` indexes `nslices` consecutive AsmRef entries, slice order.
@@ -72,8 +74,10 @@ struct cleave_plan_s {
     // assembly work list (original tasks only; reissued pieces write into their parents' blocks)
     std::vector<cleave::AsmItem> asm_items;
     std::vector<cleave::AsmRef> asm_refs;
-    struct AsmGroup { uint32_t sp, item0, n_items; };   // sp: padded slice count, 0 = scalar kernel
+    struct AsmGroup { uint32_t sp, item0, n_items, single; };   // sp: padded slice count, 0 = scalar kernel; single: one-slice GEMMs
     std::vector<AsmGroup> asm_groups;              // one launch each
+
+    bool fused = false;                            // last execution wrote one-slice GEMMs straight to C
 
     cleave::DeviceState* dev = nullptr;
 };

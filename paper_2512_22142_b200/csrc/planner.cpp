@@ -444,11 +444,11 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
 }
 
 // ---- exec work list -----------------------------------------------------------------------------
-// A task is cut into tiles of 256 rows x w columns, w <= 256 chosen so the column tiles are balanced
-// and 16-aligned (the kernel runs a tile as two 128-row halves that share the B operand).  Tiles are ordered so that tiles running at the same time share operand panels in
-// L2: by GEMM, K-range, band of 2048 rows, then column, then row.
+// A task is cut into tiles of 256 rows x 256 columns (a pair of CTAs runs one tile: 128 rows and half
+// of the columns each).  Tiles are ordered so that tiles running at the same time share operand
+// panels in L2: by GEMM, K-range, band of 4096 rows, then column, then row.
 void build_tiles(cleave_plan_s& p, uint32_t first_task) {
-    const uint32_t kBandRows = 2048;
+    const uint32_t kBandRows = 4096;
     const size_t begin = p.tiles.size();
     p.task_ntiles.resize(p.tasks.size(), 0);
     for (uint32_t id = first_task; id < p.tasks.size(); ++id) {
@@ -458,8 +458,7 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
         if ((t.k0 % 64) || ((t.k1 % 64) && t.k1 != g.K) || (g.transA && (t.m0 % 8)) || (!g.transB && (t.n0 % 8)) ||
             (g.lda % 8) || (g.ldb % 8))
             p.exec_unsupported = 1;
-        const uint32_t nt0 = (uint32_t)cdiv(beta, 256);
-        const uint32_t w = (uint32_t)(cdiv(cdiv(beta, nt0), 16) * 16);
+        const uint32_t w = 256;      // full-width tiles first, the remainder last: fewest operand bytes per FLOP
         const uint32_t nt = (uint32_t)cdiv(beta, w), mt = (uint32_t)cdiv(alpha, 256);
         p.task_ntiles[id] = nt * (uint32_t)cdiv(alpha, 128);      // bookkeeping counts 128-row half-tiles
         for (uint32_t ti = 0; ti < mt; ++ti)
@@ -467,7 +466,8 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
                 TileDesc d;
                 std::memset(&d, 0, sizeof d);
                 d.task = id; d.gemm = t.gemm;
-                d.flags = TILE_VALID | (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN);
+                d.flags = TILE_VALID | (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN) |
+                          (p.ksplit[t.gemm] == 1 ? TILE_SINGLE : 0u);
                 d.rows = std::min(256u, alpha - ti * 256);
                 d.cols = std::min(w, beta - tj * w);
                 d.n_mma = (d.cols + 15) / 16 * 16;
@@ -475,6 +475,8 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
                 d.n_col = t.n0 + tj * w;
                 d.k0 = t.k0; d.k1 = t.k1;
                 d.ld = beta;
+                d.ldc = g.N;
+                d.c_off = (uint64_t)d.m_row * g.N + d.n_col;
                 d.out_off = t.part_off + (uint64_t)ti * 256 * beta + (uint64_t)tj * w;
                 p.tiles.push_back(d);
             }
@@ -575,13 +577,14 @@ int build_assembly(cleave_plan_s& p) {
     // one launch per class: reorder the items so that each class is contiguous (GEMM order inside)
     std::vector<AsmItem> sorted;
     sorted.reserve(p.asm_items.size());
-    for (uint32_t cls : {1u, 2u, 4u, 8u, 16u, 32u, 0u}) {
-        const uint32_t item0 = (uint32_t)sorted.size();
-        for (uint32_t gi = 0; gi < p.gemms.size(); ++gi)
-            if (gemm_sp[gi] == cls)
-                sorted.insert(sorted.end(), p.asm_items.begin() + first_item[gi], p.asm_items.begin() + first_item[gi + 1]);
-        if (sorted.size() > item0) p.asm_groups.push_back({cls, item0, (uint32_t)sorted.size() - item0});
-    }
+    for (uint32_t single : {1u, 0u})
+        for (uint32_t cls : {1u, 2u, 4u, 8u, 16u, 32u, 0u}) {
+            const uint32_t item0 = (uint32_t)sorted.size();
+            for (uint32_t gi = 0; gi < p.gemms.size(); ++gi)
+                if (gemm_sp[gi] == cls && (p.ksplit[gi] == 1 ? 1u : 0u) == single)
+                    sorted.insert(sorted.end(), p.asm_items.begin() + first_item[gi], p.asm_items.begin() + first_item[gi + 1]);
+            if (sorted.size() > item0) p.asm_groups.push_back({cls, item0, (uint32_t)sorted.size() - item0, single});
+        }
     p.asm_items.swap(sorted);
     return 0;
 }

@@ -68,6 +68,9 @@ class GpuRun:
     def exec(self):
         self.plan.exec(self.A, self.B, self.partials)
 
+    def exec_fused(self):
+        self.plan.exec_fused(self.A, self.B, self.partials, self.C)
+
     def assemble(self):
         self.plan.assemble(self.partials, self.C)
 

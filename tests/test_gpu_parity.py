@@ -124,6 +124,49 @@ def test_churn_reissue_equals_no_failure():
         assert np.array_equal(out[gi], good[gi])
 
 
+def test_fused_write_out_equals_exec_plus_assemble():
+    """One-slice GEMMs written straight to C by the exec kernel: same bits as the two-step path,
+    also through a failure and its reissue."""
+    import paper_2512_22142_b200 as cl
+    w = ci.config(4, 8)
+    ts = ci.make_tensors(w)
+    p = lib_plan_for(w)
+    S = [p.ksplit(i) for i in range(p.n_gemms)]
+    assert 1 in S and max(S) > 1                      # both kinds of GEMM are present
+    base = GpuRun(w, ts, p)
+    base.exec(); base.assemble(); p.check_status()
+    good = base.results()
+
+    p2 = lib_plan_for(w)
+    run = GpuRun(w, ts, p2)                            # C starts as NaN: nothing may be left unwritten
+    launches_two_step = p2.num_launches
+    run.exec_fused(); run.assemble(); p2.check_status()
+    assert p2.num_launches < launches_two_step         # the one-slice groups are not launched any more
+    for g, a, b in zip(w.gemms, good, run.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), g.name
+
+    import torch
+    other = [torch.empty_like(c) for c in run.C]
+    with pytest.raises(cl.CleaveError) as e:           # part of the result already sits in the first C
+        p2.assemble(run.partials, other)
+    assert e.value.code == -1
+
+    failed = ci.make_failed_ids(p2.num_tasks, w.fail_frac, w.seed + 2)
+    p2.set_drops(failed)
+    for c in run.C:
+        c.fill_(float("nan"))
+    run.partials.fill_(float("nan"))
+    run.exec_fused(); run.assemble()
+    assert p2.status() == -9 and any(np.isnan(c).any() for c in run.results())
+    run.reissue(failed); run.assemble()
+    assert p2.status() == 0
+    for g, a, b in zip(w.gemms, good, run.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), g.name
+    run.exec(); run.assemble(); p2.check_status()      # a plain exec ends fused mode
+    for g, a, b in zip(w.gemms, good, run.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), g.name
+
+
 @pytest.mark.parametrize("S", [1, 2, 3, 4, 5, 8, 13])
 def test_assembly_bit_exact_vs_fp32_tree(S):
     """Random fp32 partials (not products): the assembly kernel must reproduce the balanced
