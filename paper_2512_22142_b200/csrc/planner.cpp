@@ -24,7 +24,11 @@ const uint64_t kNs = 1000000000ull;
 const uint64_t kTmax = 1ull << 50;
 
 inline uint64_t cdiv(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
-inline u128 cdiv128(u128 a, u128 b) { return (a + b - 1) / b; }
+// most numerators fit 64 bits: take the hardware division then (the 128-bit one is a library call)
+inline u128 cdiv128(u128 a, u128 b) {
+    if (!(a >> 63) && !(b >> 63)) return ((uint64_t)a + (uint64_t)b - 1) / (uint64_t)b;
+    return (a + b - 1) / b;
+}
 inline uint64_t sat64(u128 x) { return x > (u128)UINT64_MAX ? UINT64_MAX : (uint64_t)x; }
 
 // ---- cost model (Section 4.1) ---------------------------------------------------------------
@@ -355,8 +359,8 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
     std::vector<uint8_t> is_failed(p.tasks.size(), 0);
     for (uint32_t f : F) is_failed[f] = 1;
 
-    struct Round { std::vector<uint32_t> live; std::set<uint32_t> dead; std::map<uint32_t, u128> load;
-                   std::map<uint32_t, std::vector<uint32_t>> held; };
+    struct Round { std::vector<uint32_t> live; std::set<uint32_t> dead; std::vector<u128> load;   // load, held: per live[i]
+                   std::map<uint32_t, std::vector<uint32_t>> held_by_dev; std::vector<std::vector<uint32_t>> held; };
     std::map<uint32_t, Round> rounds;                     // per affected GEMM
     for (uint32_t f : F) {
         Round& r = rounds[p.tasks[f].gemm];
@@ -370,10 +374,12 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
         auto it = rounds.find(t.gemm);
         if (it == rounds.end() || (t.flags & CLEAVE_TASK_SUPERSEDED) || is_failed[t.id]) continue;
         if (it->second.dead.count(t.dev)) continue;
-        it->second.held[t.dev].push_back(t.id);
+        it->second.held_by_dev[t.dev].push_back(t.id);
     }
     for (auto& kv : rounds) {
-        for (auto& h : kv.second.held) { kv.second.live.push_back(h.first); kv.second.load[h.first] = 0; }
+        for (auto& h : kv.second.held_by_dev) {          // ascending device id
+            kv.second.live.push_back(h.first); kv.second.load.push_back(0); kv.second.held.push_back(std::move(h.second));
+        }
         if (kv.second.live.empty()) return CLEAVE_E_NO_DEVICES;
     }
 
@@ -413,26 +419,45 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
         Round& r = rounds[pc.gemm];
         const uint32_t a = pc.m1 - pc.m0, b = pc.n1 - pc.n0, kk = pc.k1 - pc.k0;
         bool found = false;
-        u128 best_cand = 0; uint64_t best_cost = 0; uint32_t best_dev = 0;
-        for (uint32_t k : r.live) {
-            const cleave_device_t& d = p.devices[k];
+        u128 best_cand = 0; uint64_t best_cost = 0; size_t best_i = 0;
+        for (size_t li = 0; li < r.live.size(); ++li) {
+            const cleave_device_t& d = p.devices[r.live[li]];
             if (mem_task(a, b, kk, o) > (u128)d.mem_bytes) continue;
-            std::vector<std::pair<uint32_t, uint32_t>> rows, cols;
-            for (uint32_t hid : r.held[k]) {
+            // rows / columns of the piece this survivor does not hold yet (its own tasks of this GEMM whose
+            // K-range contains the piece's); the common case of at most one such task needs no interval union
+            const std::vector<uint32_t>& held = r.held[li];
+            uint32_t a_hat, b_hat, n_rel = 0, last = 0;
+            for (uint32_t hid : held) {
                 const cleave_task_t& h = task_at(hid);
-                if (h.k0 <= pc.k0 && h.k1 >= pc.k1) { rows.emplace_back(h.m0, h.m1); cols.emplace_back(h.n0, h.n1); }
+                if (h.k0 <= pc.k0 && h.k1 >= pc.k1) { ++n_rel; last = hid; }
             }
-            const uint32_t a_hat = uncovered(pc.m0, pc.m1, rows), b_hat = uncovered(pc.n0, pc.n1, cols);
+            if (n_rel == 0) {
+                a_hat = a; b_hat = b;
+            } else if (n_rel == 1) {
+                const cleave_task_t& h = task_at(last);
+                const uint32_t ra = std::max(h.m0, pc.m0), rb = std::min(h.m1, pc.m1);
+                const uint32_t ca = std::max(h.n0, pc.n0), cb = std::min(h.n1, pc.n1);
+                a_hat = a - (rb > ra ? rb - ra : 0u);
+                b_hat = b - (cb > ca ? cb - ca : 0u);
+            } else {
+                std::vector<std::pair<uint32_t, uint32_t>> rows, cols;
+                for (uint32_t hid : held) {
+                    const cleave_task_t& h = task_at(hid);
+                    if (h.k0 <= pc.k0 && h.k1 >= pc.k1) { rows.emplace_back(h.m0, h.m1); cols.emplace_back(h.n0, h.n1); }
+                }
+                a_hat = uncovered(pc.m0, pc.m1, rows);
+                b_hat = uncovered(pc.n0, pc.n1, cols);
+            }
             const uint64_t c = std::max(std::max(cost_dl(a_hat, b_hat, kk, d, o.b_in, false), cost_ul(a, b, d, o.b_out)),
                                         cost_comp(a, b, kk, d));
-            const u128 cand = r.load[k] + c;
-            if (!found || cand < best_cand) { found = true; best_cand = cand; best_cost = c; best_dev = k; }
+            const u128 cand = r.load[li] + c;
+            if (!found || cand < best_cand) { found = true; best_cand = cand; best_cost = c; best_i = li; }
         }
         if (!found) return CLEAVE_E_INFEASIBLE;
-        pc.dev = best_dev;
+        pc.dev = r.live[best_i];
         pc.cost_ns = best_cost;
-        r.load[best_dev] += best_cost;
-        r.held[best_dev].push_back(pc.id);
+        r.load[best_i] += best_cost;
+        r.held[best_i].push_back(pc.id);
     }
 
     for (uint32_t f : F) p.tasks[f].flags |= CLEAVE_TASK_SUPERSEDED;

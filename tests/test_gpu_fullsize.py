@@ -11,14 +11,7 @@ from oracle import check, numerics as nm
 pytestmark = pytest.mark.gpu
 
 
-def test_config3_sampled_entries_and_freivalds():
-    import torch
-    w = ci.config(3)
-    ts = ci.make_tensors(w)
-    p = lib_plan_for(w)
-    run = GpuRun(w, ts, p)
-    run.exec(); run.assemble(); p.check_status()
-    torch.cuda.synchronize()
+def _check_against_oracle(w, ts, run, freivalds_reps=2):
     rng = np.random.default_rng(7)
     wide = {}
     for gi, g in enumerate(w.gemms):
@@ -34,5 +27,66 @@ def test_config3_sampled_entries_and_freivalds():
         got = C[rows, cols].astype(np.float64)
         assert np.all(np.abs(got - ref) <= 1e-2 * bound), g.name
         assert np.linalg.norm(got - ref) <= 1e-3 * np.linalg.norm(ref), g.name
-        worst, scale = check.freivalds_residual(A, B, C, seed=gi, reps=2)
+        worst, scale = check.freivalds_residual(A, B, C, seed=gi, reps=freivalds_reps)
         assert worst <= 1e-3 * scale, g.name     # any lost or doubled block shifts r^T C s far beyond rounding
+
+
+def test_config3_sampled_entries_and_freivalds():
+    """Llama-7B-shaped layer, 1024 devices, the launch configuration the benchmark times (fused
+    write-out of one-slice GEMMs)."""
+    import torch
+    w = ci.config(3)
+    ts = ci.make_tensors(w)
+    p = lib_plan_for(w)
+    run = GpuRun(w, ts, p)
+    run.exec_fused(); run.assemble(); p.check_status()
+    torch.cuda.synchronize()
+    _check_against_oracle(w, ts, run)
+
+
+def test_config4_churn_full_size():
+    """Same layer with 10 % of the tasks failed mid-step: the re-planned, reissued and re-assembled
+    result equals the no-failure result bit for bit and matches the oracle; the task list after the
+    re-plan equals the oracle's."""
+    import torch
+    from helpers import oracle_plan_for, task_matrix_lib, task_matrix_oracle
+    from oracle.reissue import reissue as oracle_reissue
+    w = ci.config(4)
+    ts = ci.make_tensors(w)
+    p = lib_plan_for(w)
+    run = GpuRun(w, ts, p)
+    run.exec(); run.assemble(); p.check_status()
+    torch.cuda.synchronize()
+    good = [c.clone() for c in run.C]
+    failed = ci.make_failed_ids(p.num_tasks, w.fail_frac, w.seed + 2)
+    p.set_drops(failed)
+    run.partials.fill_(float("nan"))
+    for c in run.C:
+        c.fill_(float("nan"))
+    run.exec(); run.assemble()
+    assert p.status() == -9
+    run.reissue(None)                                  # the bookkeeping finds the unfinished tasks itself
+    run.assemble()
+    assert p.status() == 0
+    torch.cuda.synchronize()
+    for g, a, b in zip(w.gemms, good, run.C):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32)), g.name
+    op = oracle_plan_for(w)
+    oracle_reissue(op, failed)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    _check_against_oracle(w, ts, run, freivalds_reps=1)
+
+
+def test_config5_sampled_entries():
+    """Llama-13B-shaped layer, 4096 devices: many small tasks, up to four K-slices."""
+    import torch
+    w = ci.config(5)
+    ts = ci.make_tensors(w)
+    p = lib_plan_for(w)
+    assert p.num_tasks > 30000 and max(p.ksplit(i) for i in range(p.n_gemms)) >= 4
+    run = GpuRun(w, ts, p)
+    run.exec_fused(); run.assemble(); p.check_status()
+    torch.cuda.synchronize()
+    done = p.done_counts()
+    assert (done == np.array([p.task_num_tiles(i) for i in range(p.num_tasks)])).all()
+    _check_against_oracle(w, ts, run, freivalds_reps=1)
