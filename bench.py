@@ -34,6 +34,21 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def measured_traffic(kernel: str):
+    """DRAM bytes per full-size launch recorded from an ncu capture (profiles/dram_traffic.txt), or
+    None when there is no record or the kernel's source changed since the counters were taken."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            rec = json.load(f)[kernel]
+        with open(os.path.join(ROOT, rec["source"]), "rb") as f:
+            if hashlib.sha1(f.read()).hexdigest() != rec["sha1"] or rec["dram_bytes_half_size_launch"] is None:
+                return None
+        return rec["dram_bytes_half_size_launch"] * rec["scale_to_full"]
+    except Exception:
+        return None
+
+
 def load_peaks():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -382,7 +397,8 @@ def run_ours(args):
             "churn": churn, "e2e_ms_per_step": e2e_ms, "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
         },
         "roofline": {"kernel": "exec_pair_kernel", "bound": "tensor", "achieved": exec_tflops, "peak": peaks["bf16_tflops_sustained"],
-                     "unit": "TFLOP/s", "frac": exec_tflops / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "unit": "TFLOP/s", "frac": exec_tflops / peaks["bf16_tflops_sustained"],
+                     "traffic": measured_traffic("exec_pair_kernel") if (args.config == 3 and args.scale == 1 and not args.two_step) else None,
                      "peak_kind": f"{peak_kind}, sustained cuBLAS bf16 (kernel timed inside a long step)",
                      "frac_of_burst": exec_tflops / peaks["bf16_tflops"], "frac_of_nominal": exec_tflops / NOMINAL_BF16_TFLOPS},
         "roofline_assemble": {"kernel": "assemble_vec_kernel", "bound": "hbm", "achieved": asm_gbs, "peak": peaks["hbm_gbs"],
