@@ -10,6 +10,7 @@
 //   widths and team heights in granules by largest remainder; cut every rectangle into its S
 //   K-slices; split whatever still violates the memory constraint.
 #include <algorithm>
+#include <array>
 #include <cstring>
 #include <map>
 #include <numeric>
@@ -414,32 +415,45 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
     auto task_at = [&](uint32_t id) -> const cleave_task_t& {
         return id < p.tasks.size() ? p.tasks[id] : pieces[id - p.tasks.size()];
     };
+    // Per GEMM and piece shape the costs that do not depend on what a survivor caches are the same for
+    // every piece of that shape: max(uplink, compute), and the full cost when nothing is cached
+    // (UINT64_MAX marks a survivor whose memory cannot hold the piece).
+    struct ShapeCost { std::vector<uint64_t> ul_comp, full; };
+    std::map<std::array<uint32_t, 4>, ShapeCost> shape_costs;
     for (uint32_t pi : order) {
         cleave_task_t& pc = pieces[pi];
         Round& r = rounds[pc.gemm];
         const uint32_t a = pc.m1 - pc.m0, b = pc.n1 - pc.n0, kk = pc.k1 - pc.k0;
+        ShapeCost& sc = shape_costs[{pc.gemm, a, b, kk}];
+        if (sc.full.empty()) {
+            sc.ul_comp.resize(r.live.size());
+            sc.full.resize(r.live.size());
+            for (size_t li = 0; li < r.live.size(); ++li) {
+                const cleave_device_t& d = p.devices[r.live[li]];
+                sc.ul_comp[li] = std::max(cost_ul(a, b, d, o.b_out), cost_comp(a, b, kk, d));
+                sc.full[li] = mem_task(a, b, kk, o) > (u128)d.mem_bytes ? UINT64_MAX
+                                                                         : std::max(cost_dl(a, b, kk, d, o.b_in, false), sc.ul_comp[li]);
+            }
+        }
         bool found = false;
         u128 best_cand = 0; uint64_t best_cost = 0; size_t best_i = 0;
         for (size_t li = 0; li < r.live.size(); ++li) {
-            const cleave_device_t& d = p.devices[r.live[li]];
-            if (mem_task(a, b, kk, o) > (u128)d.mem_bytes) continue;
+            if (sc.full[li] == UINT64_MAX) continue;
             // rows / columns of the piece this survivor does not hold yet (its own tasks of this GEMM whose
             // K-range contains the piece's); the common case of at most one such task needs no interval union
             const std::vector<uint32_t>& held = r.held[li];
-            uint32_t a_hat, b_hat, n_rel = 0, last = 0;
+            uint32_t a_hat = a, b_hat = b, n_rel = 0, last = 0;
             for (uint32_t hid : held) {
                 const cleave_task_t& h = task_at(hid);
                 if (h.k0 <= pc.k0 && h.k1 >= pc.k1) { ++n_rel; last = hid; }
             }
-            if (n_rel == 0) {
-                a_hat = a; b_hat = b;
-            } else if (n_rel == 1) {
+            if (n_rel == 1) {
                 const cleave_task_t& h = task_at(last);
                 const uint32_t ra = std::max(h.m0, pc.m0), rb = std::min(h.m1, pc.m1);
                 const uint32_t ca = std::max(h.n0, pc.n0), cb = std::min(h.n1, pc.n1);
                 a_hat = a - (rb > ra ? rb - ra : 0u);
                 b_hat = b - (cb > ca ? cb - ca : 0u);
-            } else {
+            } else if (n_rel > 1) {
                 std::vector<std::pair<uint32_t, uint32_t>> rows, cols;
                 for (uint32_t hid : held) {
                     const cleave_task_t& h = task_at(hid);
@@ -448,8 +462,9 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
                 a_hat = uncovered(pc.m0, pc.m1, rows);
                 b_hat = uncovered(pc.n0, pc.n1, cols);
             }
-            const uint64_t c = std::max(std::max(cost_dl(a_hat, b_hat, kk, d, o.b_in, false), cost_ul(a, b, d, o.b_out)),
-                                        cost_comp(a, b, kk, d));
+            const uint64_t c = (a_hat == a && b_hat == b)
+                                   ? sc.full[li]
+                                   : std::max(cost_dl(a_hat, b_hat, kk, p.devices[r.live[li]], o.b_in, false), sc.ul_comp[li]);
             const u128 cand = r.load[li] + c;
             if (!found || cand < best_cand) { found = true; best_cand = cand; best_cost = c; best_i = li; }
         }
