@@ -205,6 +205,45 @@ def test_assembly_scalar_path_bit_exact():
     assert np.array_equal(C.cpu().numpy().view(np.uint32), ref.view(np.uint32))
 
 
+@pytest.mark.parametrize("T,din,dout", [(1, 8, 8), (8, 8, 8), (130, 72, 264), (257, 64, 8), (300, 520, 136)])
+def test_degenerate_and_small_shapes_exact(T, din, dout):
+    """Smallest legal shapes (one row, K = 8), shapes below one tile, and shapes one element past a
+    tile edge, in all three operand layouts, as a single task and as a ragged 2 x 2 x 1 grid."""
+    for grid in ((1, 1, 1), (2, 2, 1)):
+        if grid[0] > min(T, din) or grid[1] > min(din, dout) or (grid != (1, 1, 1) and (din % 16 or dout % 16)):
+            continue
+        w = _custom_workload(T, [("p", din, dout)], uniform=grid)
+        w.n_devices = 0
+        _run_and_compare_exact(w)
+
+
+def test_more_slices_than_granules_and_many_devices():
+    # forced K-split larger than the number of K-granules is clamped; more devices than output cells
+    w = _custom_workload(256, [("p", 128, 256)], n_devices=40)
+    p, op, run, ref = _run_and_compare_exact(w, dict(ksplit=9))
+    assert p.ksplit(0) == 1 and p.ksplit(2) == 2          # K = 128 -> 1 granule; K = 256 -> 2 granules
+
+
+def test_bad_arguments_are_rejected_on_the_host():
+    import torch
+    import paper_2512_22142_b200 as cl
+    w = ci.config(1)
+    p = lib_plan_for(w)
+    x = torch.zeros(256, 768, dtype=torch.bfloat16, device="cuda:0")
+    wt = torch.zeros(768, 768, dtype=torch.bfloat16, device="cuda:0")
+    part = torch.zeros(p.arena_elems + 64, dtype=torch.float32, device="cuda:0")
+    c = torch.zeros(256, 768, dtype=torch.float32, device="cuda:0")
+    for bad in (lambda: p.exec([x.data_ptr() + 2], [wt], part),            # operand not 16-byte aligned
+                lambda: p.exec([0], [wt], part),                           # null operand
+                lambda: p.exec([x], [wt], part[1:]),                       # arena not 128-byte aligned
+                lambda: p.assemble(part, [c.data_ptr() + 4]),              # C not 16-byte aligned
+                lambda: p.reissue([99], [x], [wt], part)):                 # task id out of range
+        with pytest.raises(cl.CleaveError) as e:
+            bad()
+        assert e.value.code in (-1, -5)
+    p.exec([x], [wt], part); p.assemble(part, [c]); p.check_status()       # the plan is still usable afterwards
+
+
 def test_unsupported_alignment_is_rejected():
     import torch
     import paper_2512_22142_b200 as cl
