@@ -377,6 +377,23 @@ def run_ours(args):
                  "status": p2.status()}
         p2.close()
 
+    # ---- block verification (Section 6 of the paper), once, on the result of the last step -------------------
+    verify = None
+    if not args.no_verify:
+        t = plan.tasks()
+        live = (t["flags"] & 1) == 0
+        al, be, ka = (t["m1"] - t["m0"]).astype(np.float64), (t["n1"] - t["n0"]).astype(np.float64), (t["k1"] - t["k0"]).astype(np.float64)
+        vbytes = float((((al + be) * ka * 2 + al * be * 4) * live).sum())
+        plan.verify(A, B, partials, seed=1)            # first call allocates
+        v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        v0.record()
+        n_bad, _ = plan.verify(A, B, partials, seed=2)
+        v1.record()
+        torch.cuda.synchronize()
+        vms = v0.elapsed_time(v1)
+        verify = {"flagged_tasks": int(n_bad), "ms": vms, "algorithmic_GB": vbytes / 1e9, "GB_per_s": vbytes / vms / 1e6,
+                  "frac_of_measured_hbm": vbytes / vms / 1e6 / load_peaks()[0]["hbm_gbs"]}
+
     peaks, peak_kind = load_peaks()
     exec_tflops = flops / (exec_ms * 1e-3) / 1e12
     asm_gbs = asm_bytes / (asm_ms * 1e-3) / 1e9
@@ -394,7 +411,7 @@ def run_ours(args):
             "plan_ms_host": plan_ms, "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
             "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
             "pct_of_measured_sustained_bf16": 100 * value / world / peaks["bf16_tflops_sustained"],
-            "churn": churn, "e2e_ms_per_step": e2e_ms, "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
+            "churn": churn, "verify": verify, "e2e_ms_per_step": e2e_ms, "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
         },
         "roofline": {"kernel": "exec_pair_kernel", "bound": "tensor", "achieved": exec_tflops, "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": exec_tflops / peaks["bf16_tflops_sustained"],
@@ -428,6 +445,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-churn", action="store_true")
+    ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--two-step", action="store_true", help="cleave_exec + full cleave_assemble instead of the fused write-out")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -187,6 +187,26 @@ CLEAVE_API int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t
  * tasks run at the next cleave_exec.  Works without a CUDA device. */
 CLEAVE_API int cleave_replan(cleave_plan_t* p, const uint32_t* failed, uint32_t n, uint32_t* first_new);
 
+/* Verification of the returned blocks (Section 6, "Robustness to poisoning attacks": the server
+ * dispatched the inputs and received the block, so it can test it with random vectors and
+ * matrix-vector products instead of a GEMM).  For every live task t, with vectors r, s of +-1
+ * entries,   lhs = r^T P_t s   and   rhs = (A_t^T r) . (B_t s)   are compared:
+ * the task is flagged when |lhs - rhs| > tol * (|A_t^T r| . |B_t s|), or when either side is not a
+ * number (a block that was never written).  (The paper prints the right side as (A r)^T (B s); with
+ * A_t of shape alpha x kappa and r of length alpha it is read as (A_t^T r)^T (B_t s).)
+ * Entry e of vector v (0 = r, 1 = s) of task t is -1 when the top bit of SplitMix64's output
+ * function applied to seed + (t << 33 | e << 1 | v) is set, else +1.  Sums are fp32: tol = 2e-5
+ * accepts honest blocks of the benchmark layers and catches a changed entry larger than about a
+ * tenth of a typical one.  Blocks are read from `partials`, or from the C given to the last
+ * cleave_exec_fused for one-slice GEMMs.
+ *   *n_bad [host] receives the number of flagged tasks.  Synchronises the stream.  The first call
+ *   allocates.  Requires K % 4 == 0.  Errors: E_INVAL, E_UNSUPPORTED, E_CUDA, E_NOMEM. */
+CLEAVE_API int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, const float* partials,
+                             uint64_t seed, float tol, uint32_t* n_bad, void* stream);
+/* lhs, rhs, scale, flag (1.0 = flagged) of every task of the last cleave_verify, 4 floats per task,
+ * id order; superseded tasks read 0, 0, 0, 0.   out [host, 4 * number of tasks at that call]. */
+CLEAVE_API int cleave_verify_values(cleave_plan_t* p, float* out);
+
 /* Synchronises `stream` and returns the device status: 0, E_TIMEOUT or E_BOUNDS (sticky since
  * the last cleave_exec), E_INCOMPLETE (verdict of the latest cleave_assemble), or E_CUDA. */
 CLEAVE_API int cleave_status(cleave_plan_t* p, void* stream);

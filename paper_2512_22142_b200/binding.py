@@ -53,6 +53,8 @@ _sig = {
     "cleave_assemble_static": (_i, [_vp, _vp, _vp, _vp]),
     "cleave_reissue": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp]),
     "cleave_replan": (_i, [_vp, _vp, _u32, C.POINTER(_u32)]),
+    "cleave_verify": (_i, [_vp, _vp, _vp, _vp, _u64, C.c_float, C.POINTER(_u32), _vp]),
+    "cleave_verify_values": (_i, [_vp, _vp]),
     "cleave_status": (_i, [_vp, _vp]),
     "cleave_done_counts": (_i, [_vp, _vp, _vp]),
     "cleave_task_num_tiles": (_u32, [_vp, _u32]),
@@ -207,6 +209,18 @@ class Plan:
         first = C.c_uint32(0)
         _check(lib.cleave_replan(self._h, f.ctypes.data if len(f) else None, len(f), C.byref(first)), "cleave_replan")
         return first.value
+
+    def verify(self, A, B, partials, seed: int, tol: float = 2e-5, stream=None):
+        """cleave_verify + cleave_verify_values: (number of flagged tasks, float32 array [n_tasks, 4] of
+        lhs, rhs, scale, flag)."""
+        pa, pb = _ptr_array(A), _ptr_array(B)
+        bad = C.c_uint32(0)
+        n = self.num_tasks
+        _check(lib.cleave_verify(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(), seed, tol, C.byref(bad),
+                                 _stream(stream)), "cleave_verify")
+        vals = np.zeros((n, 4), dtype=np.float32)
+        _check(lib.cleave_verify_values(self._h, vals.ctypes.data), "cleave_verify_values")
+        return bad.value, vals
 
     def status(self, stream=None) -> int:
         return lib.cleave_status(self._h, _stream(stream))

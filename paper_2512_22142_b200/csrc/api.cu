@@ -32,6 +32,11 @@ struct DeviceState {
     std::vector<const void*> last_a, last_b;
     std::vector<float*> last_c;
     bool drops_dirty = true;
+    // block verification (created on first cleave_verify)
+    cleave_gemm_t* gemm_table = nullptr;
+    uint32_t* ksplit_table = nullptr;
+    const void** ab_ptrs = nullptr;
+    float4* verify_out = nullptr;     uint32_t verify_cap = 0, verify_n = 0;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};   // exec begin/end, assemble begin/end
     bool ev_exec = false, ev_asm = false;
 };
@@ -219,7 +224,8 @@ void device_state_free(DeviceState* d) {
     if (!d) return;
     cudaFree(d->tasks); cudaFree(d->tiles); cudaFree(d->dropped); cudaFree(d->done); cudaFree(d->ntiles);
     cudaFree(d->failed_ids); cudaFree(d->words); cudaFree(d->maps); cudaFree(d->asm_items); cudaFree(d->asm_refs);
-    cudaFree(d->c_ptrs); cudaFree(d->ldcs);
+    cudaFree(d->c_ptrs); cudaFree(d->ldcs); cudaFree(d->gemm_table); cudaFree(d->ksplit_table); cudaFree(d->ab_ptrs);
+    cudaFree(d->verify_out);
     for (auto& e : d->ev) if (e) cudaEventDestroy(e);
     cudaGetLastError();
     delete d;
@@ -388,6 +394,54 @@ int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t n, const v
 int cleave_replan(cleave_plan_t* p, const uint32_t* failed, uint32_t n, uint32_t* first_new) {
     if (!p || (n && !failed) || !first_new) return CLEAVE_E_INVAL;
     try { return plan_reissue(*p, failed, n, first_new); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+}
+
+int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, const float* partials, uint64_t seed,
+                  float tol, uint32_t* n_bad, void* stream) {
+    if (!p || !A || !B || !partials || !n_bad || !(tol >= 0.f)) return CLEAVE_E_INVAL;
+    for (const auto& g : p->gemms) if ((g.K % 4) || (g.lda % 8) || (g.ldb % 8)) return CLEAVE_E_UNSUPPORTED;
+    if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    DeviceState* d = p->dev;
+    const size_t n = p->gemms.size();
+    if (!d->gemm_table) {
+        RC_TRY(dev_alloc(&d->gemm_table, n)); RC_TRY(dev_alloc(&d->ksplit_table, n)); RC_TRY(dev_alloc(&d->ab_ptrs, 2 * n));
+        CU_TRY(cudaMemcpyAsync(d->gemm_table, p->gemms.data(), n * sizeof(cleave_gemm_t), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->ksplit_table, p->ksplit.data(), n * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    }
+    if (d->verify_cap < d->tasks_cap) {
+        CU_TRY(cudaStreamSynchronize(st));
+        cudaFree(d->verify_out);
+        d->verify_out = nullptr;
+        RC_TRY(dev_alloc(&d->verify_out, d->tasks_cap));
+        d->verify_cap = d->tasks_cap;
+    }
+    std::vector<const void*> ab(2 * n);
+    uint32_t sign_bytes = 0;
+    for (size_t i = 0; i < n; ++i) {
+        if (!A[i] || !B[i] || ((uintptr_t)A[i] & 15) || ((uintptr_t)B[i] & 15)) return CLEAVE_E_INVAL;
+        ab[2 * i] = A[i]; ab[2 * i + 1] = B[i];
+    }
+    for (const auto& t : p->tasks) sign_bytes = std::max(sign_bytes, (t.m1 - t.m0) + (t.n1 - t.n0));
+    sign_bytes = (sign_bytes + 15) / 16 * 16;
+    if (sign_bytes > 200 * 1024) return CLEAVE_E_UNSUPPORTED;
+    CU_TRY(cudaMemcpyAsync(d->ab_ptrs, ab.data(), ab.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemsetAsync(d->words + 3, 0, sizeof(unsigned int), st));
+    CU_TRY(launch_verify(d->tasks, d->tasks_n, d->gemm_table, d->ksplit_table, d->ab_ptrs, partials, d->c_ptrs, p->fused ? 1 : 0,
+                         seed, tol, d->verify_out, d->words + 3, sign_bytes, st));
+    d->verify_n = d->tasks_n;
+    unsigned int bad = 0;
+    CU_TRY(cudaMemcpyAsync(&bad, d->words + 3, sizeof bad, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    *n_bad = bad;
+    return 0;
+}
+
+int cleave_verify_values(cleave_plan_t* p, float* out) {
+    if (!p || !out || !p->dev || !p->dev->verify_out) return CLEAVE_E_INVAL;
+    CU_TRY(cudaMemcpy(out, p->dev->verify_out, (size_t)p->dev->verify_n * sizeof(float4), cudaMemcpyDeviceToHost));
+    return 0;
 }
 
 int cleave_status(cleave_plan_t* p, void* stream) {

@@ -46,6 +46,9 @@ cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, 
                               unsigned int* status, cudaStream_t st);
 cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
                                   uint32_t n_tasks, uint32_t* out_ids, unsigned int* out_count, cudaStream_t st);
+cudaError_t launch_verify(const cleave_task_t* tasks, uint32_t n_tasks, const cleave_gemm_t* gemms, const uint32_t* ksplit,
+                          const void* const* ab_ptrs, const float* partials, float* const* c_ptrs, int fused, uint64_t seed,
+                          float tol, float4* out, unsigned int* n_bad, uint32_t sign_bytes, cudaStream_t st);
 // sp = padded slice count of the vectorised kernel (1, 2, 4, 8, 16, 32), 0 = scalar kernel
 cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
                             const float* partials, float* const* Cptr, const uint32_t* ldcs, cudaStream_t st);

@@ -42,6 +42,8 @@ def test_config3_sampled_entries_and_freivalds():
     run.exec_fused(); run.assemble(); p.check_status()
     torch.cuda.synchronize()
     _check_against_oracle(w, ts, run)
+    bad, vals = p.verify(run.A, run.B, run.partials, seed=5)     # every returned block passes the vector check
+    assert bad == 0 and np.all(np.abs(vals[:, 0] - vals[:, 1]) <= 5e-6 * vals[:, 2] + 1e-5)
 
 
 def test_config4_churn_full_size():
