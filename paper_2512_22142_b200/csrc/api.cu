@@ -60,15 +60,31 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // 2-D bf16 tensor map over a row-major [rows x cols] matrix with row stride ld: boxes of
-// 64 (contiguous) x 64 elements, 128-byte swizzle, zero fill outside the matrix.
-int encode_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+// 64 (contiguous) x box_rows elements, 128-byte swizzle, zero fill outside the matrix.
+int encode_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return CLEAVE_E_CUDA;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {ld * 2};
-    cuuint32_t box[2] = {kBlockK, kSubRows};
+    cuuint32_t box[2] = {kBlockK, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
+}
+
+// The same matrix, whose cols are a multiple of 64, seen as [cols / 64][rows][64]: one box of
+// 64 x 64 x 2 brings two neighbouring 64-column groups (each a 64-row x 128-byte block in shared
+// memory, the second 8 KB after the first) with one TMA operation.
+int encode_map_groups(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return CLEAVE_E_CUDA;
+    cuuint64_t dims[3] = {kSubRows, rows, cols / kSubRows};
+    cuuint64_t strides[2] = {ld * 2, kSubRows * 2};
+    cuuint32_t box[3] = {kSubRows, kBlockK, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
@@ -99,7 +115,7 @@ int sync_device_state(cleave_plan_s* p, cudaStream_t st) {
         CU_TRY(exec_pair_kernel_prepare());
         RC_TRY(dev_alloc(&d->words, 4));
         CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
-        RC_TRY(dev_alloc(&d->maps, 2 * p->gemms.size()));
+        RC_TRY(dev_alloc(&d->maps, kMapsPerGemm * p->gemms.size()));
         RC_TRY(dev_alloc(&d->c_ptrs, p->gemms.size()));
         RC_TRY(dev_alloc(&d->ldcs, p->gemms.size()));
         std::vector<uint32_t> ldc;
@@ -158,13 +174,22 @@ int update_maps(cleave_plan_s* p, const void* const* A, const void* const* B, cu
     bool same = d->last_a.size() == n;
     for (size_t i = 0; same && i < n; ++i) same = (d->last_a[i] == A[i] && d->last_b[i] == B[i]);
     if (same) return 0;
-    std::vector<CUtensorMap> host(2 * n);
+    std::vector<CUtensorMap> host(kMapsPerGemm * n);
     for (size_t i = 0; i < n; ++i) {
         const cleave_gemm_t& g = p->gemms[i];
         if (!A[i] || !B[i] || ((uintptr_t)A[i] & 15) || ((uintptr_t)B[i] & 15)) return CLEAVE_E_INVAL;
         // stored shapes: A is [M x K] or, transposed, [K x M]; B is [K x N] or, transposed, [N x K]
-        RC_TRY(g.transA ? encode_map(&host[2 * i], A[i], g.K, g.M, g.lda) : encode_map(&host[2 * i], A[i], g.M, g.K, g.lda));
-        RC_TRY(g.transB ? encode_map(&host[2 * i + 1], B[i], g.N, g.K, g.ldb) : encode_map(&host[2 * i + 1], B[i], g.K, g.N, g.ldb));
+        CUtensorMap* m = &host[kMapsPerGemm * i];            // A, B with 64 x 64 boxes; A, B with double-size boxes
+        RC_TRY(g.transA ? encode_map(m + 0, A[i], g.K, g.M, g.lda, kSubRows) : encode_map(m + 0, A[i], g.M, g.K, g.lda, kSubRows));
+        RC_TRY(g.transB ? encode_map(m + 1, B[i], g.N, g.K, g.ldb, kSubRows) : encode_map(m + 1, B[i], g.K, g.N, g.ldb, kSubRows));
+        // double-size boxes: 128 rows of a K-contiguous operand, two 64-wide groups of an M/N-contiguous one
+        // (only when M / N is a multiple of 64; otherwise the slot repeats the small map and is never used)
+        if (!g.transA) RC_TRY(encode_map(m + 2, A[i], g.M, g.K, g.lda, 2 * kSubRows));
+        else if (g.M % kSubRows == 0) RC_TRY(encode_map_groups(m + 2, A[i], g.K, g.M, g.lda));
+        else m[2] = m[0];
+        if (g.transB) RC_TRY(encode_map(m + 3, B[i], g.N, g.K, g.ldb, 2 * kSubRows));
+        else if (g.N % kSubRows == 0) RC_TRY(encode_map_groups(m + 3, B[i], g.K, g.N, g.ldb));
+        else m[3] = m[1];
     }
     // pageable source: the copy is staged before the call returns, so `host` may go out of scope
     CU_TRY(cudaMemcpyAsync(d->maps, host.data(), host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, st));

@@ -19,6 +19,7 @@ constexpr uint32_t kPairABytes = 2 * kSubBytes;      // per CTA and stage: 128 r
 constexpr uint32_t kPairBBytes = 2 * kSubBytes;      // ... and half of the (<= 256) columns of B
 constexpr uint32_t kPairStageBytes = kPairABytes + kPairBBytes;   // 32768
 constexpr int kPairStages = 6;
+constexpr int kMapsPerGemm = 4;                      // A, B with 64 x 64 boxes, then A, B with double-size boxes
 constexpr int kAccSlots = 2;                         // accumulator slots in tensor memory (double buffer)
 constexpr uint32_t kAccCols = 256;
 constexpr uint32_t kTmemCols = 512;

@@ -91,6 +91,11 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap,
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const void* tmap, uint32_t bar_cluster_addr, int32_t c0, int32_t c1, int32_t c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -206,19 +211,31 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
             if (d.flags & TILE_END) break;
-            const CUtensorMap* map_a = maps + 2 * d.gemm;
+            const CUtensorMap* map_a = maps + kMapsPerGemm * d.gemm;
             const CUtensorMap* map_b = map_a + 1;
-            if (d.gemm != last_gemm) { tensormap_acquire(map_a); tensormap_acquire(map_b); last_gemm = d.gemm; }
+            if (d.gemm != last_gemm) {
+                for (int x = 0; x < kMapsPerGemm; ++x) tensormap_acquire(map_a + x);
+                last_gemm = d.gemm;
+            }
             const uint32_t half_n = d.n_mma / 2;
-            const uint32_t nsub_a = (rows_of_rank(d.rows, rank) + kSubRows - 1) / kSubRows;
-            const uint32_t nsub_b = (half_n + kSubRows - 1) / kSubRows;
+            const uint32_t my_rows = rows_of_rank(d.rows, rank);
+            const uint32_t a_x = d.m_row + rank * kBlockM, b_x = d.n_col + rank * half_n;
+            // More than 64 rows / columns of an operand come with ONE operation where a double-size box
+            // exists (fewer, larger TMA operations: +9 % on GEMMs whose operands are K-contiguous); an
+            // M/N-contiguous operand also needs its first element on a 64-element group boundary.
+            const bool a_big = (d.flags & TILE_A_BIG) && my_rows > kSubRows && (!(d.flags & TILE_A_MN) || a_x % kSubRows == 0);
+            const bool b_big = (d.flags & TILE_B_BIG) && half_n > kSubRows && (!(d.flags & TILE_B_MN) || b_x % kSubRows == 0);
+            const uint32_t nsub_a = a_big ? 1u : (my_rows + kSubRows - 1) / kSubRows;
+            const uint32_t nsub_b = b_big ? 1u : (half_n + kSubRows - 1) / kSubRows;
+            // bytes per stage do not depend on the box size: a double-size box is two 8 KB boxes
             const uint32_t tx_both = stage_bytes_of_rank(d.rows, d.n_mma, 0u) + stage_bytes_of_rank(d.rows, d.n_mma, 1u);
             const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
             const bool is_a = lane < nsub_a, is_b = !is_a && lane < nsub_a + nsub_b;
             const uint32_t j = is_a ? lane : lane - nsub_a;
-            const CUtensorMap* my_map = is_a ? map_a : map_b;
+            const bool my_big = is_a ? a_big : b_big;
+            const CUtensorMap* my_map = (is_a ? map_a : map_b) + (my_big ? 2 : 0);
             const bool my_mn = is_a ? (d.flags & TILE_A_MN) : (d.flags & TILE_B_MN);
-            const int32_t my_x = (int32_t)((is_a ? d.m_row + rank * kBlockM : d.n_col + rank * half_n) + j * kSubRows);
+            const int32_t my_x = (int32_t)((is_a ? a_x : b_x) + j * kSubRows);
             const uint32_t my_off = (is_a ? 0u : kPairABytes) + j * kSubBytes;
             for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const uint32_t s = it % kPairStages, ph = (it / kPairStages) & 1u;
@@ -229,8 +246,9 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
                 if (is_a || is_b) {
                     const uint32_t dst = stage_base + s * kPairStageBytes + my_off;
                     const uint32_t bar = full_leader0 + s * 8u;
-                    if (my_mn) tma_load_2d_pair(dst, my_map, bar, my_x, k);
-                    else       tma_load_2d_pair(dst, my_map, bar, k, my_x);
+                    if (my_mn && my_big) tma_load_3d_pair(dst, my_map, bar, 0, k, my_x / (int32_t)kSubRows);
+                    else if (my_mn)      tma_load_2d_pair(dst, my_map, bar, my_x, k);
+                    else                 tma_load_2d_pair(dst, my_map, bar, k, my_x);
                 }
             }
         }

@@ -31,7 +31,9 @@ static_assert(sizeof(TileDesc) == 64, "TileDesc must be 64 bytes");
 // A_MN / B_MN: the operand is stored with M (resp. N) contiguous (transA = 1, resp. transB = 0)
 // SINGLE: the GEMM has one K-slice, so the tile's block is already the final value of C there;
 // DIRECT: (set per launch) write it to C instead of the arena
-enum : uint32_t { TILE_VALID = 1u, TILE_END = 2u, TILE_A_MN = 4u, TILE_B_MN = 8u, TILE_SINGLE = 16u, TILE_DIRECT = 32u };
+// A_BIG / B_BIG: the operand has a tensor map with double-size boxes (one TMA operation per 128 rows or columns)
+enum : uint32_t { TILE_VALID = 1u, TILE_END = 2u, TILE_A_MN = 4u, TILE_B_MN = 8u, TILE_SINGLE = 16u, TILE_DIRECT = 32u,
+                  TILE_A_BIG = 64u, TILE_B_BIG = 128u };
 
 // One unit of assembly work: `nrows` full rows of a rectangle of C in which every K-slice is
 // served by one task.  `ref0` indexes `nslices` consecutive AsmRef entries, slice order.

@@ -507,7 +507,8 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
                 std::memset(&d, 0, sizeof d);
                 d.task = id; d.gemm = t.gemm;
                 d.flags = TILE_VALID | (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN) |
-                          (p.ksplit[t.gemm] == 1 ? TILE_SINGLE : 0u);
+                          (p.ksplit[t.gemm] == 1 ? TILE_SINGLE : 0u) |
+                          ((!g.transA || g.M % 64 == 0) ? TILE_A_BIG : 0u) | ((g.transB || g.N % 64 == 0) ? TILE_B_BIG : 0u);
                 d.rows = std::min(256u, alpha - ti * 256);
                 d.cols = std::min(w, beta - tj * w);
                 d.n_mma = (d.cols + 15) / 16 * 16;
