@@ -11,7 +11,6 @@ namespace cleave {
 
 // exec kernel geometry: a tile of <= 256 rows x <= 256 columns is run by a pair of CTAs
 constexpr uint32_t kBlockM = 128;                    // rows of a tile owned by one CTA of the pair
-constexpr uint32_t kBlockNMax = 256;                 // widest MMA N
 constexpr uint32_t kBlockK = 64;                     // K per pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kSubRows = 64;                    // rows (or M/N elements) per TMA box
 constexpr uint32_t kSubBytes = kSubRows * kBlockK * 2;          // 8192: one 64 x 64 bf16 box

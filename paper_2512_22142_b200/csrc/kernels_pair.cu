@@ -69,7 +69,10 @@ static __device__ __noinline__ bool mbar_wait_cl_slow(uint32_t bar, uint32_t par
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
+                // give up: raise the abort flag of both CTAs of the pair so that every role leaves at its next check
+                const uint32_t flag = smem_u32(const_cast<uint32_t*>(abort_flag));
+                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(flag, 0u)), "r"(1u) : "memory");
+                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(flag, 1u)), "r"(1u) : "memory");
                 atomicOr(status, STATUS_TIMEOUT);
                 return false;
             }
@@ -252,8 +255,13 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
                 }
             }
         }
-        // In-flight copies land in this CTA's shared memory: the leader's MMA thread has waited for every
-        // armed stage (or the pair is aborting and falls to the bounded cluster teardown below).
+        // Every stage armed on the normal path has been waited for by the leader's MMA thread, and a stage
+        // only completes once this CTA's own bytes have landed.  When the pair is aborting, copies may
+        // still be in flight towards this CTA's shared memory: give them a bounded time to land.
+        if (*abort_flag && lane == 0) {
+            const uint64_t t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000ull) { }
+        }
     } else if (warp == kMmaWarp) {
         // ---- MMA issuer (leader only) ---------------------------------------------------------------------------
         if (rank == 0 && lane == 0) {
