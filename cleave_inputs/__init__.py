@@ -105,6 +105,25 @@ def projection_gemms(tokens: int, projections: Sequence[Tuple[str, int, int]],
     return gemms, tensors
 
 
+def attention_gemms(n_heads: int, seq: int, d_head: int):
+    """The two GEMMs of every attention head (batch x heads of them are independent; the paper's
+    table of representative GEMMs lists Q.K^T as 1024 x 128 x 1024, count 128 x 32):
+      scores  S = Q . K^T   (M = seq, N = seq, K = d_head)   K stored [seq x d_head] -> transB = 1
+      context O = P . V     (M = seq, N = d_head, K = seq)   P stands in for softmax(S) in bf16"""
+    gemms: List[GemmSpec] = []
+    tensors: Dict[str, TensorSpec] = {}
+    for h in range(n_heads):
+        tensors[f"h{h}.Q"] = TensorSpec(seq, d_head, 1.0)
+        tensors[f"h{h}.K"] = TensorSpec(seq, d_head, 1.0)
+        tensors[f"h{h}.P"] = TensorSpec(seq, seq, 0.05)
+        tensors[f"h{h}.V"] = TensorSpec(seq, d_head, 1.0)
+    for h in range(n_heads):
+        gemms.append(GemmSpec(f"h{h}.qk", seq, seq, d_head, 0, 1, d_head, d_head, f"h{h}.Q", f"h{h}.K"))
+    for h in range(n_heads):
+        gemms.append(GemmSpec(f"h{h}.pv", seq, d_head, seq, 0, 0, seq, d_head, f"h{h}.P", f"h{h}.V"))
+    return gemms, tensors
+
+
 MB = 1 << 20
 GB = 1 << 30
 
@@ -143,6 +162,12 @@ def config(i: int, scale: int = 1) -> Workload:
         return Workload("cfg5-llama13b-layer", gemms, tensors,
                         n_devices=max(8, 4096 // (scale * scale)),
                         mem_range=(128 * MB, 2 * GB), seed=0)
+    if i == 6:
+        # not one of the five benchmark configurations: the attention GEMMs of the paper's GEMM-shape
+        # table (1024 x 128 x 1024 per head), many tiny independent GEMMs; 1024 heads at scale 1
+        gemms, tensors = attention_gemms(max(2, 1024 // (scale * scale)), s(1024, 64), s(128, 64))
+        return Workload("attention-gemms", gemms, tensors, n_devices=max(4, 64 // scale),
+                        mem_range=(256 * MB, 4 * GB), seed=0)
     raise ValueError(f"no config {i}")
 
 

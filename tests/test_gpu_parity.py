@@ -73,6 +73,16 @@ def test_scaled_configs_gaussian(cfg, scale):
     _run_and_compare_exact(w, integer=False)
 
 
+def test_attention_gemms_as_tasks():
+    """Many small independent GEMMs in one task list (scores Q.K^T and context P.V per head):
+    every GEMM has its own operands and tensor maps; K = 64 is a single K-block."""
+    w = ci.config(6, 4)                                  # 64 heads, seq 256, head dim 64: 128 GEMMs
+    assert len(w.gemms) == 128
+    _run_and_compare_exact(w, integer=True)
+    p, *_ = _run_and_compare_exact(w, integer=False)
+    assert p.num_tasks >= 2 * len(w.gemms)
+
+
 def test_scaled_config2_integer_exact():
     _run_and_compare_exact(ci.config(2, 4), integer=True)
 
