@@ -254,6 +254,26 @@ def test_bad_arguments_are_rejected_on_the_host():
     p.exec([x], [wt], part); p.assemble(part, [c]); p.check_status()       # the plan is still usable afterwards
 
 
+def test_every_task_dropped():
+    """Nothing to run: the kernel's scheduler finds no runnable tile, the bookkeeping reports every
+    task unfinished, and with every device dead no re-plan exists."""
+    import paper_2512_22142_b200 as cl
+    w = ci.config(2, 8)
+    ts = ci.make_tensors(w)
+    p = lib_plan_for(w)
+    p.set_drops(np.arange(p.num_tasks))
+    run = GpuRun(w, ts, p)
+    run.exec(); run.assemble()
+    assert p.status() == -9 and p.done_counts().sum() == 0
+    assert all(np.isnan(c).all() for c in run.results())
+    with pytest.raises(cl.CleaveError) as e:
+        run.reissue(None)
+    assert e.value.code == -4                             # E_NO_DEVICES
+    p.set_drops([])
+    run.exec(); run.assemble(); p.check_status()
+    assert all(np.isfinite(c).all() for c in run.results())
+
+
 def test_unsupported_alignment_is_rejected():
     import torch
     import paper_2512_22142_b200 as cl
