@@ -224,7 +224,7 @@ int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, uint32_t
               int clear_status, float* partials, cudaStream_t st) {
     DeviceState* d = p->dev;
     CU_TRY(launch_arm_queue(d->tiles, tile_begin, tile_end, d->tasks, d->dropped, d->done, task_begin, task_end,
-                            d->words + 0, d->words + 1, clear_status, p->fused ? 1 : 0, st));
+                            d->words + 0, d->words + 1, clear_status, p->fused ? 1 : 0, p->arena_elems, st));
     if (tile_end > tile_begin) {
         // one cluster of two CTAs per pair of SMs, never more clusters than tiles
         const uint32_t clusters = std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)d->sm_count / 2, tile_end - tile_begin));
@@ -318,10 +318,10 @@ uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm) { return (p &
 uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->makespan.size()) ? p->makespan[gemm] : 0; }
 uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->tstar.size()) ? p->tstar[gemm] : 0; }
 uint32_t cleave_plan_num_tiles(const cleave_plan_t* p) { return p ? (uint32_t)p->tiles.size() : 0; }
-// exec: arm + grouped GEMM; assemble: clear verdict + bookkeeping check + one kernel per slice-count class
+
 uint32_t cleave_plan_num_launches(const cleave_plan_t* p) {
     if (!p) return 0;
-    uint32_t n = 4;
+    uint32_t n = 5;          // clear + arm + exec, clear verdict + bookkeeping check, then the assembly kernels
     for (const auto& grp : p->asm_groups) if (!(p->fused && grp.single)) ++n;
     return n;
 }

@@ -17,16 +17,17 @@
 
 namespace cleave {
 
+__global__ void clear_status_bits_kernel(unsigned int* status, unsigned int mask) { *status &= ~mask; }
+
 // -------------------------------------------------------------------------------------------------
 // arm_queue_kernel
 // -------------------------------------------------------------------------------------------------
 __global__ void arm_queue_kernel(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
                                  const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                                 unsigned int* ticket, unsigned int* status, int clear_status, int direct) {
+                                 unsigned int* ticket, unsigned int* status, int direct, unsigned long long arena_elems) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         *ticket = tile_begin;
-        if (clear_status) *status = 0;
     }
     const uint32_t t = tile_begin + i;
     if (t < tile_end) {
@@ -35,6 +36,11 @@ __global__ void arm_queue_kernel(TileDesc* tiles, uint32_t tile_begin, uint32_t 
         uint32_t f = tiles[t].flags & ~(uint32_t)(TILE_VALID | TILE_DIRECT);
         if (!skip) f |= TILE_VALID;
         if (direct && (f & TILE_SINGLE)) f |= TILE_DIRECT;
+        // range check of the block the tile will write: a tile that would leave the arena is not run
+        if (!(f & TILE_DIRECT) && tiles[t].out_off + (unsigned long long)(tiles[t].rows - 1) * tiles[t].ld + tiles[t].cols > arena_elems) {
+            f &= ~(uint32_t)TILE_VALID;
+            atomicOr(status, STATUS_BOUNDS);
+        }
         tiles[t].flags = f;
     }
     const uint32_t k = task_begin + i;
@@ -44,7 +50,6 @@ __global__ void arm_queue_kernel(TileDesc* tiles, uint32_t tile_begin, uint32_t 
 // -------------------------------------------------------------------------------------------------
 // bookkeeping kernels
 // -------------------------------------------------------------------------------------------------
-__global__ void clear_status_bits_kernel(unsigned int* status, unsigned int mask) { *status &= ~mask; }
 
 __global__ void check_done_kernel(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
                                   uint32_t n_tasks, unsigned int* status) {
@@ -168,12 +173,15 @@ __global__ void assemble_scalar_kernel(const AsmItem* __restrict__ items, const 
 // -------------------------------------------------------------------------------------------------
 cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
                              const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, cudaStream_t st) {
+                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, uint64_t arena_elems,
+                             cudaStream_t st) {
     uint32_t n = tile_end - tile_begin;
     if (task_end - task_begin > n) n = task_end - task_begin;
     if (n == 0) n = 1;
+    // a fresh execution forgets the verdicts of the previous one (before the arming threads may raise new ones)
+    if (clear_status) clear_status_bits_kernel<<<1, 1, 0, st>>>(status, 0xFFFFFFFFu);
     arm_queue_kernel<<<(n + 255) / 256, 256, 0, st>>>(tiles, tile_begin, tile_end, tasks, dropped, done, task_begin,
-                                                       task_end, ticket, status, clear_status, direct);
+                                                       task_end, ticket, status, direct, (unsigned long long)arena_elems);
     return cudaGetLastError();
 }
 

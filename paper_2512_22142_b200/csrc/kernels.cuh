@@ -37,7 +37,8 @@ enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BOUNDS = 2u, STATUS_INCOMPLETE
 
 cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
                              const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, cudaStream_t st);
+                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, uint64_t arena_elems,
+                             cudaStream_t st);
 cudaError_t exec_pair_kernel_prepare();
 cudaError_t launch_exec_pair(uint32_t clusters, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
                              const CUtensorMap* maps, float* partials, float* const* c_ptrs, uint32_t* done,
