@@ -115,3 +115,16 @@ def test_uniform_and_errors(cl):
     with pytest.raises(cl.CleaveError) as e:
         cl.plan(w.gemms, tiny)
     assert e.value.code == -3                                    # E_INFEASIBLE
+
+
+def test_header_is_plain_c_and_defaults_agree_with_oracle(cl, tmp_path):
+    import subprocess
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "cleave.h"\nint main(void) { cleave_plan_opts_t o; cleave_task_t t; (void)o; (void)t; '
+                   'return sizeof(cleave_task_t) == 64 && sizeof(cleave_device_t) == 48 && sizeof(cleave_gemm_t) == 24 ? 0 : 1; }\n')
+    exe = tmp_path / "use_header"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    assert subprocess.run([str(exe)]).returncode == 0
+    o, ref = cl.default_opts(), Opts()
+    for name in ("gran_m", "gran_n", "gran_k", "kslice_max", "ksplit", "ksplit_cap", "reissue_fanout", "b_in", "b_out"):
+        assert getattr(o, name) == getattr(ref, name), name
