@@ -254,6 +254,27 @@ def test_bad_arguments_are_rejected_on_the_host():
     p.exec([x], [wt], part); p.assemble(part, [c]); p.check_status()       # the plan is still usable afterwards
 
 
+def test_new_operand_buffers_and_side_stream():
+    """The same plan run on other operand buffers (the tensor maps must follow the pointers) and on
+    a stream other than the default one."""
+    import torch
+    w = ci.config(2, 8)
+    p, op = lib_plan_for(w), oracle_plan_for(w)
+    side = torch.cuda.Stream()
+    for seed in (0, 1):
+        ts = ci.make_tensors(w, seed=seed, integer=True)
+        A, B = oracle_operands(w, ts)
+        ref = nm.assemble(op, nm.execute(op, A, B))
+        run = GpuRun(w, ts, p)                           # fresh device tensors: new addresses
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            run.exec_fused(); run.assemble()
+        side.synchronize()
+        p.check_status()
+        for g, got, want in zip(w.gemms, run.results(), ref):
+            assert np.array_equal(got.astype(np.float64), want), (seed, g.name)
+
+
 def test_every_task_dropped():
     """Nothing to run: the kernel's scheduler finds no runnable tile, the bookkeeping reports every
     task unfinished, and with every device dead no re-plan exists."""
