@@ -360,8 +360,10 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
     std::vector<uint8_t> is_failed(p.tasks.size(), 0);
     for (uint32_t f : F) is_failed[f] = 1;
 
-    struct Round { std::vector<uint32_t> live; std::set<uint32_t> dead; std::vector<u128> load;   // load, held: per live[i]
-                   std::map<uint32_t, std::vector<uint32_t>> held_by_dev; std::vector<std::vector<uint32_t>> held; };
+    struct Span { uint32_t m0, m1, n0, n1, k0, k1; };
+    struct Round { std::vector<uint32_t> live; std::set<uint32_t> dead; std::vector<u128> load;   // load, held, first: per live[i]
+                   std::map<uint32_t, std::vector<uint32_t>> held_by_dev; std::vector<std::vector<uint32_t>> held;
+                   std::vector<Span> first; };                   // ranges of held[i][0]: most survivors hold one task
     std::map<uint32_t, Round> rounds;                     // per affected GEMM
     for (uint32_t f : F) {
         Round& r = rounds[p.tasks[f].gemm];
@@ -380,6 +382,8 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
     for (auto& kv : rounds) {
         for (auto& h : kv.second.held_by_dev) {          // ascending device id
             kv.second.live.push_back(h.first); kv.second.load.push_back(0); kv.second.held.push_back(std::move(h.second));
+            const cleave_task_t& t0 = p.tasks[kv.second.held.back()[0]];
+            kv.second.first.push_back(Span{t0.m0, t0.m1, t0.n0, t0.n1, t0.k0, t0.k1});
         }
         if (kv.second.live.empty()) return CLEAVE_E_NO_DEVICES;
     }
@@ -442,18 +446,22 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
             // rows / columns of the piece this survivor does not hold yet (its own tasks of this GEMM whose
             // K-range contains the piece's); the common case of at most one such task needs no interval union
             const std::vector<uint32_t>& held = r.held[li];
-            uint32_t a_hat = a, b_hat = b, n_rel = 0, last = 0;
-            for (uint32_t hid : held) {
-                const cleave_task_t& h = task_at(hid);
-                if (h.k0 <= pc.k0 && h.k1 >= pc.k1) { ++n_rel; last = hid; }
+            uint32_t a_hat = a, b_hat = b, n_rel = 0;
+            if (held.size() == 1) {                          // the usual case, served from the inline copy
+                const Span& h = r.first[li];
+                if (h.k0 <= pc.k0 && h.k1 >= pc.k1) {
+                    const uint32_t ra = std::max(h.m0, pc.m0), rb = std::min(h.m1, pc.m1);
+                    const uint32_t ca = std::max(h.n0, pc.n0), cb = std::min(h.n1, pc.n1);
+                    a_hat = a - (rb > ra ? rb - ra : 0u);
+                    b_hat = b - (cb > ca ? cb - ca : 0u);
+                }
+            } else {
+                for (uint32_t hid : held) {
+                    const cleave_task_t& h = task_at(hid);
+                    if (h.k0 <= pc.k0 && h.k1 >= pc.k1) ++n_rel;
+                }
             }
-            if (n_rel == 1) {
-                const cleave_task_t& h = task_at(last);
-                const uint32_t ra = std::max(h.m0, pc.m0), rb = std::min(h.m1, pc.m1);
-                const uint32_t ca = std::max(h.n0, pc.n0), cb = std::min(h.n1, pc.n1);
-                a_hat = a - (rb > ra ? rb - ra : 0u);
-                b_hat = b - (cb > ca ? cb - ca : 0u);
-            } else if (n_rel > 1) {
+            if (n_rel >= 1) {
                 std::vector<std::pair<uint32_t, uint32_t>> rows, cols;
                 for (uint32_t hid : held) {
                     const cleave_task_t& h = task_at(hid);
