@@ -12,6 +12,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The C-ABI library is built in-tree; (re)build it when a source is newer than the binary."""
+    from paper_2512_22142_b200.build import build_library
+    build_library()
+
+
 def read_golden(name):
     """key = value lines of a fixture under tests/golden/ ('#' starts a comment)."""
     out = {}
