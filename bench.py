@@ -240,11 +240,12 @@ def run_ours(args):
     import numpy as np
     import torch
 
-    import cleave_inputs as ci
-    import paper_2512_22142_b200 as cl
-
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        from paper_2512_22142_b200.build import build_library
+        build_library()                               # no-op when the in-tree library is up to date
+    import cleave_inputs as ci
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
@@ -254,6 +255,8 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()                                # rank 0 may have just built the library
+    import paper_2512_22142_b200 as cl
 
     w = ci.config(args.config, args.scale)
     opts = {}
