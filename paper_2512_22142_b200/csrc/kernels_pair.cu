@@ -12,12 +12,14 @@
 // Synchronisation between the two CTAs uses only mbarriers:
 //   full[s]      leader's barrier; the leader's producer arms it with the bytes of BOTH CTAs, and
 //                the peer's TMA loads complete their bytes on it (cta_group::2 loads)
-//   empty[s]     in both CTAs; the leader's MMA thread commits to both at once (multicast commit)
-//   acc_full[a]  in both CTAs, multicast commit;   acc_empty[a]  leader's, both CTAs' epilogue warps
+//   empty[s]     in both CTAs; the leader's MMA thread commits to both at once (one tcgen05.commit
+//                with a two-CTA mask)
+//   acc_full[a]  in both CTAs, same two-CTA commit;   acc_empty[a]  leader's, both CTAs' epilogue warps
 //   sched ring   the leader's scheduler warp pops the ticket, writes the tile descriptor into both
 //                CTAs' slot rings and arrives on both CTAs' sched_full; every consumer of either
 //                CTA arrives on the leader's sched_empty
-// No TMA load uses cluster multicast.
+// Every TMA load is an ordinary load into the issuing CTA's own shared memory (no load is shared
+// between CTAs).
 //
 // Every device-side wait is bounded: when a wait expires the CTA records E_TIMEOUT in the status
 // word and raises its abort flag, all its roles leave their loops, the MMAs in flight are drained
