@@ -152,3 +152,52 @@ def test_helpers():
     assert split_counts(11, 3) == [4, 4, 3]
     r = r_mem(10 ** 6, 100, 2, 4)
     assert 2 * r * 100 * 2 + r * r * 4 <= 10 ** 6 < 2 * (r + 1) * 100 * 2 + (r + 1) ** 2 * 4
+
+
+def _guillotine_partitions(r0, r1, c0, c1, max_parts):
+    """All ways to cut the granule rectangle [r0,r1) x [c0,c1) into at most max_parts rectangles by
+    recursive straight cuts (every exact tiling of so small a grid is of this kind)."""
+    out = [[(r0, r1, c0, c1)]]
+    if max_parts < 2:
+        return out
+    for cut in range(r0 + 1, r1):
+        for k in range(1, max_parts):
+            for a in _guillotine_partitions(r0, cut, c0, c1, k):
+                for b in _guillotine_partitions(cut, r1, c0, c1, max_parts - len(a)):
+                    out.append(a + b)
+    for cut in range(c0 + 1, c1):
+        for k in range(1, max_parts):
+            for a in _guillotine_partitions(r0, r1, c0, cut, k):
+                for b in _guillotine_partitions(r0, r1, cut, c1, max_parts - len(a)):
+                    out.append(a + b)
+    return out
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_heuristic_is_within_a_small_factor_of_the_exhaustive_optimum(seed):
+    """Not a pin of optimality (the paper's solver is unavailable), but a guard against an absurd
+    plan: on instances small enough to enumerate every assignment of rectangles to devices
+    (one K-slice, one rectangle per device, idle devices allowed), the heuristic's makespan stays
+    within 2x of the best possible one."""
+    from itertools import permutations
+    from oracle.cost import task_cost
+    rng = np.random.default_rng(500 + seed)
+    Mg, Ng = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    g = 32
+    D = int(rng.integers(1, 4))
+    devs = small_devices(D, 900 + seed, 1 << 24, 1 << 26)
+    K = 64
+    o = Opts(gran_m=g, gran_n=g, gran_k=g, kslice_max=0, ksplit=1)
+    p = plan([Gemm(Mg * g, Ng * g, K)], devs, o)
+    best = None
+    seen = set()
+    for part in _guillotine_partitions(0, Mg, 0, Ng, D):
+        key = tuple(sorted(part))
+        if key in seen:
+            continue
+        seen.add(key)
+        for owners in permutations(range(D), len(part)):
+            cost = max(task_cost((r1 - r0) * g, (c1 - c0) * g, K, devs[k], o.b_in, o.b_out)
+                       for (r0, r1, c0, c1), k in zip(part, owners))
+            best = cost if best is None else min(best, cost)
+    assert best is not None and best <= p.makespan_ns[0] <= 2 * best
