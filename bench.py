@@ -320,6 +320,7 @@ def run_ours(args):
     total_ms = max_over_ranks(begin.elapsed_time(end))
     exec_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     asm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    step_times = [e[0].elapsed_time(e[2]) for e in ev]
     ms_per_step = total_ms / args.steps
     value = job_throughput(flops, world, ms_per_step)
 
@@ -468,7 +469,7 @@ def run_ours(args):
             "write_out": "two-step" if args.two_step else "fused for one-slice GEMMs",
             "l2": "not flushed; operands + arena + outputs per step (~%.1f GB) far exceed the 126 MB L2" %
                   ((h2d + plan.arena_elems * 4 + d2h) / 1e9),
-            "plan_ms_host": plan_ms, "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
+            "plan_ms_host": plan_ms, "step_ms_median": statistics.median(step_times), "step_ms_best": min(step_times), "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
             "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
             "pct_of_measured_sustained_bf16": 100 * value / world / peaks["bf16_tflops_sustained"],
             "churn": churn, "verify": verify, "e2e_ms_per_step": e2e_ms, "e2e_serial_ms_per_step": e2e_serial_ms,
