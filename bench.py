@@ -5,8 +5,8 @@
 
 A step is one pass of the path over one batch of synthetic input: queue arming, the grouped
 sub-GEMM execution of every task of every GEMM of the layer, and the assembly of the K-split
-partial blocks into the GEMM results.  The plan is made once before the loop (the paper solves the
-schedule once per device set and reuses it); its time and the churn path (drop 10 % of the tasks,
+partial blocks into the GEMM results.  The plan is made once before the loop (the paper computes a
+schedule when the device set changes, not per batch); its time and the churn path (drop 10 % of the tasks,
 re-plan, reissue, re-assemble) are measured separately and reported inside `config`.
 
 One JSON line is printed by rank 0.  With --gpus N > 1 (launched through torch.distributed.run)

@@ -129,7 +129,8 @@ CLEAVE_API uint32_t cleave_plan_num_tiles(const cleave_plan_t* p);        /* wor
 CLEAVE_API uint32_t cleave_plan_num_launches(const cleave_plan_t* p);     /* kernels launched by one
                                    cleave_exec[_fused] + cleave_assemble, in the current mode    */
 
-/* Host-made failures (Section 3.2, "Device departures are detected via disconnect events"): the
+/* Host-made failures (Section 3.2, scheduling workflow: a device that leaves is noticed through its
+ * broken connection and its unfinished outputs are found in the server's bookkeeping): the
  * listed tasks are skipped by every later cleave_exec / cleave_reissue launch, as if their device
  * had left before returning its block.  Replaces the previous list; n = 0 clears it.
  * ids [host, n].  Errors: E_RANGE. */
@@ -149,8 +150,8 @@ CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* c
                 void* stream);
 
 /* cleave_exec with the write-out of one-slice GEMMs fused into the sub-GEMM kernel.  For a GEMM
- * with a single K-slice a device's block is already a finished block of O (Section 4.1, "each
- * device computes A' o B', a subset of O_s"; the paper's own formulation), so the kernel stores it
+ * with a single K-slice a device's block is already a finished block of O (Section 4.1, search
+ * space of a GEMM: every device returns a block of the output; the paper's own formulation), so the kernel stores it
  * at its place in C_g instead of the arena and the following cleave_assemble has nothing to do for
  * that GEMM; GEMMs with several K-slices go through the arena as in cleave_exec.  The results are
  * bit-identical to cleave_exec + cleave_assemble.
@@ -161,8 +162,8 @@ CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* c
 CLEAVE_API int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
                                  float* const* C, void* stream);
 
-/* Parameter-server aggregation (Section 3.1 / 3.2: the server "aggregates the computed outputs";
- * with a K-split it is a sum): C_g[i,j] = sum over the K-slices s of the partial block covering
+/* Parameter-server aggregation (Section 3.1 / 3.2: the server collects the devices' output blocks
+ * into the GEMM result; with a K-split collecting means summing): C_g[i,j] = sum over the K-slices s of the partial block covering
  * (i,j) in slice s, as a balanced pairwise tree over adjacent slices padded with +0.0 to a power
  * of two -- a fixed order, so the result is deterministic.
  *   partials [device]; C [host array of n_gemms device pointers], C_g fp32 row-major, ld = N.

@@ -1,7 +1,7 @@
 """Independent checkers for plans and results (test infrastructure).
 
-Coverage: Section 4.1 requires the shards to cover the output "without redundant work"; the sum
-of areas is necessary but not sufficient for a tiling, so coverage is checked directly.
+Coverage: Section 4.1 requires the shards to cover the whole output with no work done twice; its
+sum-of-areas condition is necessary but not sufficient for a tiling, so coverage is checked directly.
 Constraints: Eq. (zero-task-constraint), Eq. (memory-constraint).
 Freivalds: Section 6 ("Robustness to poisoning attacks"): r^T (A B) s = (A^T r)^T (B s).
 """

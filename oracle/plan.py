@@ -295,7 +295,8 @@ def _finish(plan: Plan, per_gemm_rects):
 
 def plan(gemms: Sequence[Gemm], devices: Sequence[Device], opts: Opts = Opts()) -> Plan:
     """Every GEMM is planned independently over the same device list (each GEMM is its own
-    dispatch round; the decision is solved once per device set and reused, Section 3.2)."""
+    dispatch round; a schedule is computed when the device set changes and kept until it changes
+    again, Section 3.2)."""
     p = Plan(list(gemms), list(devices), opts)
     per_gemm = []
     for g in gemms:
