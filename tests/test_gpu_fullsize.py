@@ -92,3 +92,19 @@ def test_config5_sampled_entries():
     done = p.done_counts()
     assert (done == np.array([p.task_num_tiles(i) for i in range(p.num_tasks)])).all()
     _check_against_oracle(w, ts, run, freivalds_reps=1)
+
+
+def test_config2_every_output_against_the_full_oracle():
+    """GPT-2-small-shaped layer at full size (12 GEMMs, 64 devices, 0.35 TFLOP): small enough for the
+    oracle to compute every block, so every output element is compared, not a sample."""
+    from helpers import assert_within_tolerance, oracle_operands, oracle_plan_for, task_matrix_lib, task_matrix_oracle
+    w = ci.config(2)
+    ts = ci.make_tensors(w)
+    p, op = lib_plan_for(w), oracle_plan_for(w)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    A, B = oracle_operands(w, ts)
+    ref = nm.assemble(op, nm.execute(op, A, B))
+    run = GpuRun(w, ts, p)
+    run.exec_fused(); run.assemble(); p.check_status()
+    for g, got, want, a, b in zip(w.gemms, run.results(), ref, A, B):
+        assert_within_tolerance(got, want, nm.abs_bound(a, b), what=g.name)
