@@ -201,3 +201,200 @@ def test_heuristic_is_within_a_small_factor_of_the_exhaustive_optimum(seed):
                        for (r0, r1, c0, c1), k in zip(part, owners))
             best = cost if best is None else min(best, cost)
     assert best is not None and best <= p.makespan_ns[0] <= 2 * best
+
+
+# ---------------------------------------------------------------------------------- capacity and T*
+# The water-fill capacity a_k(T) is a closed form that follows from the cost terms of Section 4.1
+# (pinned in test_oracle_cost.py on the paper's worked example) and the memory constraint.  It is
+# pinned here three ways: hand-computed areas on devices where exactly one term binds, agreement
+# with a brute-force search that only calls the cost functions, and the defining property of each
+# term (the returned area is affordable within T, the next larger one is not).
+
+from oracle.cost import c_comp, c_dl, c_ul
+
+BIG = 10 ** 15
+CAP_OPTS = Opts(gran_m=1, gran_n=1, gran_k=1)
+
+
+def _one_binding_term_devices():
+    """(device, T, kappa_hat, hand-computed area, name of the binding term)"""
+    return [
+        # downlink: (T - L^d) W^d / (1e9 * kappa * b_in) = 2e6 * 1e6 / (1e9 * 200) = 10 rows + columns -> 5 x 5
+        (Device(BIG, BIG, 10 ** 6, BIG, 1000, 0), 1000 + 2 * 10 ** 6, 100, 25, "dl"),
+        # an odd budget of rows + columns: 11 -> 5 x 6
+        (Device(BIG, BIG, 10 ** 6, BIG, 1000, 0), 1000 + 22 * 10 ** 5, 100, 30, "dl"),
+        # uplink: (T - L^u) W^u / (1e9 * b_out) = 1e5 * 1e6 / 4e9 = 25 outputs
+        (Device(BIG, BIG, BIG, 10 ** 6, 0, 500), 500 + 10 ** 5, 100, 25, "ul"),
+        # compute: T F / (2000 kappa) = 1e5 * 1000 / 2e5 = 500 outputs  (F = 1000 MFLOP/s)
+        (Device(BIG, 1000, BIG, BIG, 0, 0), 10 ** 5, 100, 500, "comp"),
+        # memory: 2 r kappa b_in + r^2 b_out <= 4500 -> r = 10 (4400), r = 11 needs 4884
+        (Device(4500, BIG, BIG, BIG, 0, 0), 10 ** 5, 100, 100, "mem"),
+    ]
+
+
+@pytest.mark.parametrize("case", range(5))
+def test_capacity_hand_computed_one_binding_term(case):
+    dev, T, kappa, want, which = _one_binding_term_devices()[case]
+    assert capacity(dev, T, kappa, CAP_OPTS) == want
+    # the latency is paid before the first byte: at T = L nothing can be done yet
+    if which == "dl":
+        assert capacity(dev, dev.dl_lat_ns, kappa, CAP_OPTS) == 0
+        # long before the latency has passed the (negative) time left must not turn into an area
+        late = dev._replace(dl_lat_ns=10 ** 7)
+        assert capacity(late, 10, kappa, CAP_OPTS) == 0 and capacity(late, 10 ** 7 - 1, kappa, CAP_OPTS) == 0
+        assert capacity(dev, T - 1, kappa, CAP_OPTS) < want          # T is the first instant the area fits
+    if which == "ul":
+        assert capacity(dev, dev.ul_lat_ns, kappa, CAP_OPTS) == 0
+        assert capacity(dev, T - 1, kappa, CAP_OPTS) == want - 1
+    if which == "comp":
+        # depth matters: twice the slice depth halves the affordable area
+        assert capacity(dev, T, 2 * kappa, CAP_OPTS) == want // 2
+    if which == "mem":
+        assert capacity(dev, 10 * T, kappa, CAP_OPTS) == want          # time does not help
+
+
+def _capacity_bruteforce(dev, T, kappa, o, limit=40):
+    """min over the four terms of the largest area that term alone allows, found by trying blocks
+    with the cost functions themselves: every (alpha, beta) up to `limit` for the downlink (its cost
+    depends on alpha + beta), every 1 x n block for uplink and compute (their cost depends on the
+    area only), every square for the memory constraint."""
+    best = {"dl": 0, "ul": 0, "comp": 0}
+    for a in range(1, limit + 1):
+        for b in range(1, limit + 1):
+            if c_dl(a, b, kappa, dev, o.b_in) <= T:
+                best["dl"] = max(best["dl"], a * b)
+    for n in range(1, limit * limit + 1):
+        if c_ul(1, n, dev, o.b_out) <= T:
+            best["ul"] = n
+        if c_comp(1, n, kappa, dev) <= T:
+            best["comp"] = n
+    r = 0
+    while task_mem(r + 1, r + 1, kappa, o.b_in, o.b_out) <= dev.mem_bytes:
+        r += 1
+    area = min(best["dl"], best["ul"], best["comp"], r * r)
+    return area if area >= o.gran_m * o.gran_n else 0
+
+
+def test_capacity_equals_bruteforce_over_the_cost_functions():
+    stats = {"compared": 0, "working": 0}
+    for seed in range(10):
+        _compare_capacity_with_bruteforce(np.random.default_rng(40 + seed), stats)
+    assert stats["compared"] >= 200 and stats["working"] >= 50     # idle and working instants both occur
+
+
+def _compare_capacity_with_bruteforce(rng, stats):
+    kappa = int(rng.integers(1, 64))
+    # rates chosen so that the affordable block stays well inside the brute-force search window
+    dev = Device(int(rng.integers(2_000, 40_000)), int(rng.integers(50, 2_000)), int(rng.integers(10 ** 5, 10 ** 7)),
+                 int(rng.integers(10 ** 5, 10 ** 7)), int(rng.integers(0, 3_000)), int(rng.integers(0, 3_000)))
+    o = Opts(gran_m=int(rng.integers(1, 4)), gran_n=int(rng.integers(1, 4)), gran_k=1)
+    # instants from 0 up to where a cost term reaches the edge of the brute-force search window
+    limit = 40
+
+    def clipped(T):
+        return (c_dl(limit, limit + 1, kappa, dev, o.b_in) <= T or c_ul(1, limit * limit, dev, o.b_out) <= T or
+                c_comp(1, limit * limit, kappa, dev) <= T)
+    t_hi = 1
+    while not clipped(2 * t_hi):
+        t_hi *= 2
+    for T in [int(x) for x in rng.integers(0, t_hi, 40)] + [dev.dl_lat_ns, dev.ul_lat_ns, dev.dl_lat_ns + 1]:
+        if clipped(T):
+            continue
+        got = capacity(dev, T, kappa, o)
+        assert got == _capacity_bruteforce(dev, T, kappa, o, limit), (T, kappa, dev)
+        stats["compared"] += 1
+        stats["working"] += got > 0
+
+
+def test_capacity_defining_property_at_config_scale():
+    """On the synthetic devices of the Llama-7B-shaped workload: the square block of the returned
+    area is affordable within T under every cost term, and for the term that binds, one more
+    row + column (downlink) or one more output (uplink, compute) is not."""
+    w = ci.config(3)
+    devs = devices_from_array(ci.workload_devices(w))[:64]
+    o = Opts(gran_m=128, gran_n=128, gran_k=128)
+    kappa = 4096
+    for T in (30_000_000, 400_000_000, 3_000_000_000):
+        for d in devs:
+            a = capacity(d, T, kappa, o)
+            if a == 0:
+                continue
+            side = isqrt_(a)
+            assert c_dl(side, side, kappa, d, o.b_in) <= T
+            assert c_ul(side, side, d, o.b_out) <= T and c_ul(1, a, d, o.b_out) <= T
+            assert c_comp(side, side, kappa, d) <= T and c_comp(1, a, kappa, d) <= T
+            assert task_mem(side, side, kappa, o.b_in, o.b_out) <= d.mem_bytes
+            # which term binds: the one whose own maximum equals the returned area
+            s = 0 if T <= d.dl_lat_ns else ((T - d.dl_lat_ns) * d.dl_Bps) // (10 ** 9 * kappa * o.b_in)
+            binding = []
+            if (s // 2) * (s - s // 2) == a:
+                binding.append("dl")
+                assert c_dl(s // 2, s - s // 2, kappa, d, o.b_in) <= T < c_dl(s // 2, s - s // 2 + 1, kappa, d, o.b_in)
+            if c_ul(1, a + 1, d, o.b_out) > T:
+                binding.append("ul")
+            if c_comp(1, a + 1, kappa, d) > T:
+                binding.append("comp")
+            r = r_mem(d.mem_bytes, kappa, o.b_in, o.b_out)
+            if r * r == a:
+                binding.append("mem")
+                assert task_mem(r + 1, r + 1, kappa, o.b_in, o.b_out) > d.mem_bytes
+            assert binding, (d, T, a)
+
+
+def isqrt_(x):
+    from math import isqrt
+    return isqrt(x)
+
+
+def test_t_star_two_devices_by_hand():
+    """Water-fill level of a 20 x 20 x 100 GEMM (one slice, 400 outputs) on two compute-bound
+    devices of 1000 and 3000 MFLOP/s: a_k(T) = floor(T F_k / 2e5), so 400 outputs need
+    T (1000 + 3000) / 2e5 >= 400 up to the two floors: T = 20000 ns gives 100 + 300 exactly and
+    T = 19999 gives 99 + 299."""
+    devs = [Device(BIG, 1000, BIG, BIG, 0, 0), Device(BIG, 3000, BIG, BIG, 0, 0)]
+    o = Opts(gran_m=1, gran_n=1, gran_k=1, kslice_max=0, ksplit=1)
+    p = plan([Gemm(20, 20, 100)], devs, o)
+    assert p.t_star == [20000]
+    assert capacity(devs[0], 20000, 100, o) + capacity(devs[1], 20000, 100, o) == 400
+    assert capacity(devs[0], 19999, 100, o) + capacity(devs[1], 19999, 100, o) == 398
+    # with a downlink latency of 7000 ns on the fast device and a link that makes the downlink bind:
+    # s = floor((T - 7000) * 1e9 / (1e9 * 200)) rows + columns on device 1, compute bound on device 0
+    devs2 = [Device(BIG, 1000, BIG, BIG, 0, 0), Device(BIG, BIG, 10 ** 9, BIG, 7000, 0)]
+    p2 = plan([Gemm(20, 20, 100)], devs2, o)
+    T = p2.t_star[0]
+
+    def total(t):
+        s = 0 if t <= 7000 else (t - 7000) // 200
+        return (t * 1000) // 200000 + (s // 2) * (s - s // 2)
+    assert total(T) >= 400 > total(T - 1)
+    # at 14400: s = 37 -> 18 * 19 = 342, plus floor(14400 / 200) = 72 -> 414; at 14399: s = 36 -> 324 + 71 = 395
+    assert T == 14400
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_t_star_is_the_least_feasible_level_by_linear_scan(seed):
+    rng = np.random.default_rng(70 + seed)
+    D = int(rng.integers(1, 5))
+    devs = [Device(int(rng.integers(20_000, 200_000)), int(rng.integers(200, 2_000)), int(rng.integers(10 ** 6, 10 ** 7)),
+                   int(rng.integers(10 ** 6, 10 ** 7)), int(rng.integers(0, 2_000)), int(rng.integers(0, 2_000)))
+            for _ in range(D)]
+    o = Opts(gran_m=2, gran_n=2, gran_k=4, kslice_max=0, ksplit=1)
+    g = Gemm(int(rng.integers(4, 14)), int(rng.integers(4, 14)), int(rng.integers(4, 32)))
+    try:
+        p = plan([g], devs, o)
+    except PlanError:
+        pytest.skip("infeasible draw")
+    kappa = min(g.K, o.gran_k * -(-g.K // o.gran_k))
+    need = g.M * g.N
+    T = p.t_star[0]
+    assert sum(capacity(d, T, kappa, o) for d in devs) >= need
+    # no earlier instant suffices: the capacities (pinned above) never decrease with T, checked here on
+    # a scan of the instants below T* together with the sum itself
+    step = max(1, T // 3000)
+    prev = 0
+    for t in list(range(0, T, step)) + [T - 1]:
+        tot = sum(capacity(d, t, kappa, o) for d in devs)
+        assert tot < need
+        if t < T - 1 or t % step == 0:
+            assert tot >= prev
+            prev = tot
