@@ -45,6 +45,8 @@ class GemmSpec:
     ldb: int
     a_key: str
     b_key: str
+    level: int = 0                         # DAG level: a GEMM may read what lower levels produced
+    out_key: Optional[str] = None          # name under which the (bf16) result feeds higher levels
 
     @property
     def flops(self) -> int:
@@ -69,6 +71,7 @@ class Workload:
     fail_frac: float = 0.0
     seed: int = 0
     note: str = ""
+    produced: Dict[str, TensorSpec] = field(default_factory=dict)   # tensors written by GEMMs of the step
 
     @property
     def flops(self) -> int:
@@ -122,6 +125,26 @@ def attention_gemms(n_heads: int, seq: int, d_head: int):
     for h in range(n_heads):
         gemms.append(GemmSpec(f"h{h}.pv", seq, d_head, seq, 0, 0, seq, d_head, f"h{h}.P", f"h{h}.V"))
     return gemms, tensors
+
+
+def two_branch_chain(tokens: int, d0: int, d1: int, d2: int):
+    """A three-level DAG in the shape of a transformer block's dependencies (Section 4.1: GEMMs of a
+    level are independent, the outputs of a level are the inputs of the next):
+      level 0   Ha = X . Wa,  Hb = X . Wb          (two GEMMs sharing X, like the QKV projections)
+      level 1   Ya = Ha . Va, Yb = Hb . Vb          (each reads one level-0 output as its A operand)
+      level 2   G  = Ha^T . Hb                      (reads two level-0 outputs; contraction over tokens)
+    Produced tensors are bf16, as a training step would keep its activations."""
+    tensors = {"X": TensorSpec(tokens, d0, 1.0), "Wa": TensorSpec(d0, d1, 0.05), "Wb": TensorSpec(d0, d1, 0.05),
+               "Va": TensorSpec(d1, d2, 0.05), "Vb": TensorSpec(d1, d2, 0.05)}
+    produced = {"Ha": TensorSpec(tokens, d1, 0.0), "Hb": TensorSpec(tokens, d1, 0.0)}
+    gemms = [
+        GemmSpec("Ha", tokens, d1, d0, 0, 0, d0, d1, "X", "Wa", 0, "Ha"),
+        GemmSpec("Hb", tokens, d1, d0, 0, 0, d0, d1, "X", "Wb", 0, "Hb"),
+        GemmSpec("Ya", tokens, d2, d1, 0, 0, d1, d2, "Ha", "Va", 1, None),
+        GemmSpec("Yb", tokens, d2, d1, 0, 0, d1, d2, "Hb", "Vb", 1, None),
+        GemmSpec("G", d1, d1, tokens, 1, 0, d1, d1, "Ha", "Hb", 2, None),
+    ]
+    return gemms, tensors, produced
 
 
 MB = 1 << 20

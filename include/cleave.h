@@ -62,12 +62,15 @@ typedef struct {
  *   transA = 0: A stored [M x K], lda >= K.   transA = 1: stored [K x M], A[i,k] = X[k,i], lda >= M.
  *   transB = 0: B stored [K x N], ldb >= N.   transB = 1: stored [N x K], B[k,j] = W[j,k], ldb >= K.
  * Forward X.W is (0,0), data gradient dY.W^T is (0,1), weight gradient X^T.dY is (1,0).
- * lda, ldb in elements.  M, N, K < 2^31. */
+ * lda, ldb in elements.  M, N, K < 2^31.
+ * level: the GEMM's level in the DAG of the training step (Section 4.1, "Problem definition and
+ * objective": GEMMs of one level are independent, a level starts when the level before it has
+ * finished).  0 for a flat list.  At most 4096 levels. */
 typedef struct {
     uint32_t M, N, K;
     uint32_t lda, ldb;
     uint8_t  transA, transB;
-    uint8_t  pad_[2];
+    uint16_t level;
 } cleave_gemm_t;
 
 /* One sub-GEMM task: P[alpha x beta] = A[m0:m1, k0:k1] . B[k0:k1, n0:n1]   (alpha = m1-m0 ...).
@@ -87,7 +90,7 @@ typedef struct {
 
 /* Planner options.  Zero-initialise and call cleave_plan_opts_default. */
 typedef struct {
-    uint32_t gran_m, gran_n, gran_k;  /* block granularity in rows / columns / K (256, 128, 128) */
+    uint32_t gran_m, gran_n, gran_k;  /* block granularity in rows / columns / K (128, 128, 128) */
     uint32_t kslice_max;              /* deepest K-slice, 0 = never split for depth (default 4096)*/
     uint32_t ksplit;                  /* 0 = automatic, else the forced number of K-slices        */
     uint32_t ksplit_cap;              /* upper limit of the automatic choice (default 8)          */
@@ -126,6 +129,15 @@ CLEAVE_API uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm);  
 CLEAVE_API uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm);  /* modelled, max load  */
 CLEAVE_API uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm);     /* water-fill level    */
 CLEAVE_API uint32_t cleave_plan_num_tiles(const cleave_plan_t* p);        /* work units of the exec kernel  */
+/* Level-wise cost of Section 4.1 (equation "level-cost-s"): the modelled time of a level is that of
+ * its slowest GEMM, and levels add up.  cleave_plan_level_makespan_ns: max over the GEMMs of `level`
+ * of cleave_plan_makespan_ns (0 for an empty level); cleave_plan_step_makespan_ns: the sum over all
+ * levels, the modelled time of the distributed GEMMs of the step. */
+/* 1 if the exec kernel can sum the K-slices of this GEMM itself (CLEAVE_EXEC_FINISH), else 0. */
+CLEAVE_API uint32_t cleave_plan_finishable(const cleave_plan_t* p, uint32_t gemm);
+CLEAVE_API uint32_t cleave_plan_num_levels(const cleave_plan_t* p);
+CLEAVE_API uint64_t cleave_plan_level_makespan_ns(const cleave_plan_t* p, uint32_t level);
+CLEAVE_API uint64_t cleave_plan_step_makespan_ns(const cleave_plan_t* p);
 CLEAVE_API uint32_t cleave_plan_num_launches(const cleave_plan_t* p);     /* kernels launched by one
                                    cleave_exec[_fused] + cleave_assemble, in the current mode    */
 
@@ -153,7 +165,7 @@ CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* c
  * with a single K-slice a device's block is already a finished block of O (Section 4.1, search
  * space of a GEMM: every device returns a block of the output; the paper's own formulation), so the kernel stores it
  * at its place in C_g instead of the arena and the following cleave_assemble has nothing to do for
- * that GEMM; GEMMs with several K-slices go through the arena as in cleave_exec.  The results are
+ * that GEMM; for GEMMs with several K-slices see CLEAVE_EXEC_FINISH below.  The results are
  * bit-identical to cleave_exec + cleave_assemble.
  *   C [host array of n_gemms device pointers, fp32 row-major, ld = N, 16-byte aligned].  The same C
  *   must be passed to the cleave_assemble that follows; cleave_reissue after a fused execution writes
@@ -162,13 +174,44 @@ CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* c
 CLEAVE_API int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
                                  float* const* C, void* stream);
 
+/* The general form of the two calls above.  flags (any combination):
+ *   CLEAVE_EXEC_DIRECT  blocks of GEMMs with one K-slice are stored at their place in C (as in
+ *                       cleave_exec_fused);
+ *   CLEAVE_EXEC_FINISH  in a GEMM with several K-slices the block of a cell that is written last
+ *                       sums the cell -- every K-slice's block of that cell, read back from the
+ *                       arena -- in the fixed tree order of cleave_assemble and stores the sums in C,
+ *                       so the server-side aggregation (Section 3.2) needs no pass of its own.  Which
+ *                       block comes last changes nothing in the sums: they are bit-identical to
+ *                       cleave_assemble's.  Every block is still written to the arena.  GEMMs whose
+ *                       K-slices are cut into unequal blocks (after a memory repair), with more than
+ *                       8 K-slices or with N % 4 != 0 are left to cleave_assemble; so is every GEMM
+ *                       when a task is dropped, and after a cleave_reissue;
+ *   CLEAVE_EXEC_BF16    C holds bf16: every value written to C, by this call and by the
+ *                       cleave_assemble / cleave_reissue that follow it, is the fp32 value rounded to
+ *                       nearest even (ld = N elements, 16-byte aligned).  Arena blocks stay fp32.
+ * cleave_exec_fused is DIRECT | FINISH.  C may be NULL when neither DIRECT nor FINISH is given.
+ * level_begin, level_end: only GEMMs with level_begin <= level < level_end run (0, UINT32_MAX: all).
+ * Levels run in order inside one launch: a tile of level s starts only after every block of the
+ * levels below s (of this launch) has been written, so with DIRECT | FINISH a GEMM may take as A
+ * or B what a GEMM of a lower level wrote to its C (bf16) in the same call.  A level that lost a
+ * task leaves its output incomplete: after cleave_reissue has replayed it (and cleave_assemble, if
+ * the GEMM has several K-slices), run the higher levels again with level_begin.
+ * Errors: as cleave_exec. */
+#define CLEAVE_EXEC_DIRECT 1u
+#define CLEAVE_EXEC_FINISH 2u
+#define CLEAVE_EXEC_BF16   4u
+CLEAVE_API int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
+                                void* const* C, uint32_t flags, uint32_t level_begin, uint32_t level_end, void* stream);
+
 /* Parameter-server aggregation (Section 3.1 / 3.2: the server collects the devices' output blocks
  * into the GEMM result; with a K-split collecting means summing): C_g[i,j] = sum over the K-slices s of the partial block covering
  * (i,j) in slice s, as a balanced pairwise tree over adjacent slices padded with +0.0 to a power
  * of two -- a fixed order, so the result is deterministic.
  *   partials [device]; C [host array of n_gemms device pointers], C_g fp32 row-major, ld = N.
  * If a task that feeds C never finished, the device status becomes E_INCOMPLETE (see
- * cleave_status); the sums are still written.  At most 32 K-slices (else E_UNSUPPORTED). */
+ * cleave_status); the sums are still written.  At most 32 K-slices (else E_UNSUPPORTED).
+ * What the last execution already wrote to C (see cleave_exec_opts) is not computed again; after an
+ * execution with CLEAVE_EXEC_BF16 every C_g holds bf16. */
 CLEAVE_API int cleave_assemble(cleave_plan_t* p, const float* partials, float* const* C, void* stream);
 
 /* Churn recovery (Section 4.2): the failed tasks' devices are dead for their GEMM; every failed
@@ -217,6 +260,12 @@ CLEAVE_API int cleave_status(cleave_plan_t* p, void* stream);
  * cleave_task_num_tiles. */
 CLEAVE_API int cleave_done_counts(cleave_plan_t* p, uint32_t* done, void* stream);
 CLEAVE_API uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task);
+
+/* Bound, in nanoseconds, of every wait inside the exec kernel (default 2 s).  When a wait runs out
+ * the kernel gives up in an orderly way -- its roles leave their loops, tensor-core work in flight
+ * is drained, the status becomes E_TIMEOUT -- and the call returns; the plan stays usable.  For
+ * tests of that path: with 0 the first wait that is not satisfied at once gives up. */
+CLEAVE_API int cleave_set_wait_limit_ns(cleave_plan_t* p, uint64_t ns);
 
 /* Device time of the last exec-kernel and assembly-kernel launches on this plan, in
  * milliseconds, measured with CUDA events on the launching stream (synchronises those events). */

@@ -22,6 +22,16 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
+def f64_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bf16 (8 significant bits), ties to even, in ONE rounding from fp64; the
+    bit patterns as uint16.  (Going through fp32 first would round twice.)  Values are assumed to lie
+    in bf16's normal range or to be zero, as every output of the workloads here does."""
+    x = np.asarray(x, dtype=np.float64)
+    m, e = np.frexp(x)                       # x = m * 2^e, 0.5 <= |m| < 1
+    r = np.ldexp(np.rint(m * 256.0), e - 8)  # rint rounds half to even: 8 significant bits kept
+    return (r.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
 def op_a(stored: np.ndarray, transA: int) -> np.ndarray:
     """A as an [M x K] array.  transA = 1: stored is [K x M] and A[i, k] = stored[k, i]."""
     return stored.T if transA else stored
@@ -80,18 +90,21 @@ def assemble(plan: Plan, arena: np.ndarray, dtype=np.float64) -> List[np.ndarray
 
     Only original tasks are read: a reissued piece writes into its parent's block, so the arena
     layout never changes.  `dtype=np.float32` emulates the GPU's fp32 adds bit for bit."""
-    out = []
+    return [assemble_gemm(plan, arena, gi, dtype) for gi in range(len(plan.gemms))]
+
+
+def assemble_gemm(plan: Plan, arena: np.ndarray, gi: int, dtype=np.float64) -> np.ndarray:
+    """`assemble` for one GEMM of the plan."""
     arena = arena.astype(dtype, copy=False)
-    for gi, g in enumerate(plan.gemms):
-        S = plan.ksplit[gi]
-        slabs = [np.full((g.M, g.N), np.nan, dtype=dtype) for _ in range(S)]
-        for t in plan.tasks[:plan.n_original]:
-            if t.gemm != gi:
-                continue
-            blk = arena[t.part_off:t.part_off + t.alpha * t.beta].reshape(t.alpha, t.beta)
-            slabs[t.kslice][t.m0:t.m1, t.n0:t.n1] = blk
-        out.append(tree_sum(slabs))
-    return out
+    g = plan.gemms[gi]
+    S = plan.ksplit[gi]
+    slabs = [np.full((g.M, g.N), np.nan, dtype=dtype) for _ in range(S)]
+    for t in plan.tasks[:plan.n_original]:
+        if t.gemm != gi:
+            continue
+        blk = arena[t.part_off:t.part_off + t.alpha * t.beta].reshape(t.alpha, t.beta)
+        slabs[t.kslice][t.m0:t.m1, t.n0:t.n1] = blk
+    return tree_sum(slabs)
 
 
 def gemm_direct(A: np.ndarray, B: np.ndarray) -> np.ndarray:

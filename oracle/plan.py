@@ -54,7 +54,7 @@ class Gemm:
 
 @dataclass(frozen=True)
 class Opts:
-    gran_m: int = 256
+    gran_m: int = 128
     gran_n: int = 128
     gran_k: int = 128
     kslice_max: int = 4096

@@ -20,7 +20,7 @@ lib = C.CDLL(lib_path)
 DEVICE_DTYPE = np.dtype([(n, "<u8") for n in
                          ("mem_bytes", "flops_mflops", "dl_Bps", "ul_Bps", "dl_lat_ns", "ul_lat_ns")])
 GEMM_DTYPE = np.dtype([("M", "<u4"), ("N", "<u4"), ("K", "<u4"), ("lda", "<u4"), ("ldb", "<u4"),
-                       ("transA", "u1"), ("transB", "u1"), ("pad_", "u1", (2,))])
+                       ("transA", "u1"), ("transB", "u1"), ("level", "<u2")])
 TASK_DTYPE = np.dtype([(n, "<u4") for n in
                        ("id", "gemm", "dev", "parent", "m0", "m1", "n0", "n1", "k0", "k1", "kslice", "flags")]
                       + [("part_off", "<u8"), ("cost_ns", "<u8")])
@@ -46,6 +46,12 @@ _sig = {
     "cleave_plan_tstar_ns": (_u64, [_vp, _u32]),
     "cleave_plan_num_tiles": (_u32, [_vp]),
     "cleave_plan_num_launches": (_u32, [_vp]),
+    "cleave_plan_num_levels": (_u32, [_vp]),
+    "cleave_plan_finishable": (_u32, [_vp, _u32]),
+    "cleave_plan_level_makespan_ns": (_u64, [_vp, _u32]),
+    "cleave_plan_step_makespan_ns": (_u64, [_vp]),
+    "cleave_exec_opts": (_i, [_vp, _vp, _vp, _vp, _vp, _u32, _u32, _u32, _vp]),
+    "cleave_set_wait_limit_ns": (_i, [_vp, _u64]),
     "cleave_set_drops": (_i, [_vp, _vp, _u32]),
     "cleave_exec": (_i, [_vp, _vp, _vp, _vp, _vp]),
     "cleave_exec_fused": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
@@ -65,6 +71,9 @@ _sig = {
 for _name, (_res, _args) in _sig.items():
     _f = getattr(lib, _name)
     _f.restype, _f.argtypes = _res, _args
+
+
+EXEC_DIRECT, EXEC_FINISH, EXEC_BF16 = 1, 2, 4
 
 
 def strerror(code: int) -> str:
@@ -98,7 +107,7 @@ def gemm_array(gemms: Sequence) -> np.ndarray:
         return np.ascontiguousarray(gemms)
     a = np.zeros(len(gemms), dtype=GEMM_DTYPE)
     for i, g in enumerate(gemms):
-        a[i] = (g.M, g.N, g.K, g.lda, g.ldb, g.transA, g.transB, (0, 0))
+        a[i] = (g.M, g.N, g.K, g.lda, g.ldb, g.transA, g.transB, getattr(g, "level", 0))
     return a
 
 
@@ -185,6 +194,33 @@ class Plan:
         pa, pb, pc = _ptr_array(A), _ptr_array(B), _ptr_array(Cs)
         _check(lib.cleave_exec_fused(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(), pc.ctypes.data,
                                      _stream(stream)), "cleave_exec_fused")
+
+    def exec_opts(self, A, B, partials, Cs=None, direct=False, finish=False, bf16=False, level_begin=0,
+                  level_end=0xFFFFFFFF, stream=None) -> None:
+        """cleave_exec_opts: flags CLEAVE_EXEC_DIRECT / FINISH / BF16 and a range of DAG levels."""
+        pa, pb = _ptr_array(A), _ptr_array(B)
+        pc = _ptr_array(Cs) if Cs is not None else None
+        flags = (EXEC_DIRECT if direct else 0) | (EXEC_FINISH if finish else 0) | (EXEC_BF16 if bf16 else 0)
+        _check(lib.cleave_exec_opts(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(),
+                                    pc.ctypes.data if pc is not None else None, flags, level_begin, level_end,
+                                    _stream(stream)), "cleave_exec_opts")
+
+    def set_wait_limit_ns(self, ns: int) -> None:
+        _check(lib.cleave_set_wait_limit_ns(self._h, int(ns)), "cleave_set_wait_limit_ns")
+
+    def finishable(self, gemm: int) -> bool:
+        return bool(lib.cleave_plan_finishable(self._h, gemm))
+
+    @property
+    def num_levels(self) -> int:
+        return lib.cleave_plan_num_levels(self._h)
+
+    def level_makespan_ns(self, level: int) -> int:
+        return lib.cleave_plan_level_makespan_ns(self._h, level)
+
+    @property
+    def step_makespan_ns(self) -> int:
+        return lib.cleave_plan_step_makespan_ns(self._h)
 
     def assemble(self, partials, Cs, stream=None) -> None:
         pc = _ptr_array(Cs)

@@ -27,11 +27,16 @@ struct DeviceState {
     CUtensorMap* maps = nullptr;
     AsmItem* asm_items = nullptr;
     AsmRef* asm_refs = nullptr;
-    float** c_ptrs = nullptr;
+    void** c_ptrs = nullptr;
     uint32_t* ldcs = nullptr;
+    uint32_t* fin_ref0 = nullptr;     // cells of the in-kernel K-slice sum
+    FinRef* fin_refs = nullptr;
+    unsigned int* fin_count = nullptr;    // per cell and 32-row strip: blocks arrived in this execution
+    unsigned int* level_left = nullptr;   // per DAG level: strips still to finish in this launch
     std::vector<const void*> last_a, last_b;
-    std::vector<float*> last_c;
+    std::vector<void*> last_c;
     bool drops_dirty = true;
+    bool tiles_dirty = false;         // the host tile list was re-ordered: send it again in full
     // block verification (created on first cleave_verify)
     cleave_gemm_t* gemm_table = nullptr;
     uint32_t* ksplit_table = nullptr;
@@ -99,33 +104,48 @@ int dev_alloc(T** p, size_t n) {
 #define CU_TRY(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return CLEAVE_E_CUDA; } } while (0)
 #define RC_TRY(x) do { int rc_ = (x); if (rc_) return rc_; } while (0)
 
+// First use of a plan on a device: the mirrors that never grow.  The state is attached to the plan
+// only when every step has succeeded.
+int create_device_state(cleave_plan_s* p, cudaStream_t st, DeviceState* d) {
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return CLEAVE_E_CUDA; }
+    CU_TRY(cudaGetDevice(&d->device));
+    CU_TRY(cudaDeviceGetAttribute(&d->sm_count, cudaDevAttrMultiProcessorCount, d->device));
+    int cc_major = 0;
+    CU_TRY(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, d->device));
+    if (cc_major != 10) return CLEAVE_E_UNSUPPORTED;
+    CU_TRY(exec_pair_kernel_prepare());
+    const size_t ng = p->gemms.size();
+    RC_TRY(dev_alloc(&d->words, 4));
+    CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
+    RC_TRY(dev_alloc(&d->maps, kMapsPerGemm * ng));
+    RC_TRY(dev_alloc(&d->c_ptrs, ng));
+    RC_TRY(dev_alloc(&d->ldcs, ng));
+    std::vector<uint32_t> ldc;
+    for (auto& g : p->gemms) ldc.push_back(g.N);
+    CU_TRY(cudaMemcpyAsync(d->ldcs, ldc.data(), ldc.size() * 4, cudaMemcpyHostToDevice, st));
+    RC_TRY(dev_alloc(&d->asm_items, p->asm_items.size()));
+    RC_TRY(dev_alloc(&d->asm_refs, p->asm_refs.size()));
+    CU_TRY(cudaMemcpyAsync(d->asm_items, p->asm_items.data(), p->asm_items.size() * sizeof(AsmItem), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(d->asm_refs, p->asm_refs.data(), p->asm_refs.size() * sizeof(AsmRef), cudaMemcpyHostToDevice, st));
+    RC_TRY(dev_alloc(&d->fin_ref0, p->fin_ref0.size()));
+    RC_TRY(dev_alloc(&d->fin_refs, p->fin_refs.size()));
+    RC_TRY(dev_alloc(&d->fin_count, 4 * p->fin_ref0.size()));
+    RC_TRY(dev_alloc(&d->level_left, p->n_levels));
+    CU_TRY(cudaMemcpyAsync(d->fin_ref0, p->fin_ref0.data(), p->fin_ref0.size() * 4, cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(d->fin_refs, p->fin_refs.data(), p->fin_refs.size() * sizeof(FinRef), cudaMemcpyHostToDevice, st));
+    for (auto& e : d->ev) CU_TRY(cudaEventCreate(&e));
+    return 0;
+}
+
 // Creates the mirrors on first use and brings the growing tables (tasks, tiles) up to date.
 int sync_device_state(cleave_plan_s* p, cudaStream_t st) {
     if (!p->dev) {
-        int ndev = 0;
-        if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return CLEAVE_E_CUDA; }
         DeviceState* d = new (std::nothrow) DeviceState();
         if (!d) return CLEAVE_E_NOMEM;
+        const int rc = create_device_state(p, st, d);
+        if (rc) { cudaStreamSynchronize(st); device_state_free(d); return rc; }
         p->dev = d;
-        CU_TRY(cudaGetDevice(&d->device));
-        CU_TRY(cudaDeviceGetAttribute(&d->sm_count, cudaDevAttrMultiProcessorCount, d->device));
-        int cc_major = 0;
-        CU_TRY(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, d->device));
-        if (cc_major != 10) return CLEAVE_E_UNSUPPORTED;
-        CU_TRY(exec_pair_kernel_prepare());
-        RC_TRY(dev_alloc(&d->words, 4));
-        CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
-        RC_TRY(dev_alloc(&d->maps, kMapsPerGemm * p->gemms.size()));
-        RC_TRY(dev_alloc(&d->c_ptrs, p->gemms.size()));
-        RC_TRY(dev_alloc(&d->ldcs, p->gemms.size()));
-        std::vector<uint32_t> ldc;
-        for (auto& g : p->gemms) ldc.push_back(g.N);
-        CU_TRY(cudaMemcpyAsync(d->ldcs, ldc.data(), ldc.size() * 4, cudaMemcpyHostToDevice, st));
-        RC_TRY(dev_alloc(&d->asm_items, p->asm_items.size()));
-        RC_TRY(dev_alloc(&d->asm_refs, p->asm_refs.size()));
-        CU_TRY(cudaMemcpyAsync(d->asm_items, p->asm_items.data(), p->asm_items.size() * sizeof(AsmItem), cudaMemcpyHostToDevice, st));
-        CU_TRY(cudaMemcpyAsync(d->asm_refs, p->asm_refs.data(), p->asm_refs.size() * sizeof(AsmRef), cudaMemcpyHostToDevice, st));
-        for (auto& e : d->ev) CU_TRY(cudaEventCreate(&e));
     }
     DeviceState* d = p->dev;
     const uint32_t nt = (uint32_t)p->tasks.size(), nl = (uint32_t)p->tiles.size();
@@ -160,6 +180,7 @@ int sync_device_state(cleave_plan_s* p, cudaStream_t st) {
         cudaFree(d->tiles);
         d->tiles = tiles; d->tiles_cap = cap;
     }
+    if (d->tiles_dirty) { d->tiles_n = 0; d->tiles_dirty = false; }
     if (nl > d->tiles_n) {
         CU_TRY(cudaMemcpyAsync(d->tiles + d->tiles_n, p->tiles.data() + d->tiles_n, (nl - d->tiles_n) * sizeof(TileDesc),
                                cudaMemcpyHostToDevice, st));
@@ -209,27 +230,40 @@ int check_exec_args(cleave_plan_s* p, const void* const* A, const void* const* B
     return 0;
 }
 
-int upload_c_ptrs(cleave_plan_s* p, float* const* C, cudaStream_t st) {
+int upload_c_ptrs(cleave_plan_s* p, void* const* C, cudaStream_t st) {
     DeviceState* d = p->dev;
     const size_t n = p->gemms.size();
     for (size_t i = 0; i < n; ++i) if (!C[i] || ((uintptr_t)C[i] & 15)) return CLEAVE_E_INVAL;
     if (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin())) {
         d->last_c.assign(C, C + n);
-        CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(float*), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(void*), cudaMemcpyHostToDevice, st));
     }
     return 0;
 }
 
-int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, uint32_t task_begin, uint32_t task_end,
-              int clear_status, float* partials, cudaStream_t st) {
+// One launch of the arming kernel and the exec kernel over the work-list range [tile_begin, tile_end).
+// `fresh`: a whole execution (the arrival counters of the in-kernel K-slice sums start at zero).
+int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, bool fresh, uint32_t level_begin, uint32_t level_end,
+              float* partials, cudaStream_t st) {
     DeviceState* d = p->dev;
-    CU_TRY(launch_arm_queue(d->tiles, tile_begin, tile_end, d->tasks, d->dropped, d->done, task_begin, task_end,
-                            d->words + 0, d->words + 1, clear_status, p->fused ? 1 : 0, p->arena_elems, st));
+    CU_TRY(cudaMemsetAsync(d->level_left, 0, p->n_levels * sizeof(unsigned int), st));
+    if (fresh && !p->fin_ref0.empty()) CU_TRY(cudaMemsetAsync(d->fin_count, 0, 4 * p->fin_ref0.size() * sizeof(unsigned int), st));
+    ArmParams a;
+    a.tiles = d->tiles; a.tile_begin = tile_begin; a.tile_end = tile_end;
+    a.tasks = d->tasks; a.dropped = d->dropped; a.done = d->done;
+    a.ticket = d->words + 0; a.status = d->words + 1; a.level_left = d->level_left;
+    a.mode = p->mode; a.level_begin = level_begin; a.level_end = level_end; a.arena_elems = p->arena_elems;
+    CU_TRY(launch_arm_queue(a, fresh ? 1 : 0, st));
     if (tile_end > tile_begin) {
         // one cluster of two CTAs per pair of SMs, never more clusters than tiles
         const uint32_t clusters = std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)d->sm_count / 2, tile_end - tile_begin));
+        ExecParams e;
+        e.tiles = d->tiles; e.tile_end = tile_end; e.ticket = d->words + 0; e.maps = d->maps; e.partials = partials;
+        e.c_ptrs = d->c_ptrs; e.done = d->done; e.status = d->words + 1;
+        e.fin_ref0 = d->fin_ref0; e.fin_refs = d->fin_refs; e.fin_count = d->fin_count; e.level_left = d->level_left;
+        e.mode = p->mode; e.wait_limit_ns = p->wait_limit_ns;
         CU_TRY(cudaEventRecord(d->ev[0], st));
-        CU_TRY(launch_exec_pair(clusters, d->tiles, tile_end, d->words + 0, d->maps, partials, d->c_ptrs, d->done, d->words + 1, st));
+        CU_TRY(launch_exec_pair(clusters, e, st));
         CU_TRY(cudaEventRecord(d->ev[1], st));
         d->ev_exec = true;
     }
@@ -249,7 +283,8 @@ void device_state_free(DeviceState* d) {
     if (!d) return;
     cudaFree(d->tasks); cudaFree(d->tiles); cudaFree(d->dropped); cudaFree(d->done); cudaFree(d->ntiles);
     cudaFree(d->failed_ids); cudaFree(d->words); cudaFree(d->maps); cudaFree(d->asm_items); cudaFree(d->asm_refs);
-    cudaFree(d->c_ptrs); cudaFree(d->ldcs); cudaFree(d->gemm_table); cudaFree(d->ksplit_table); cudaFree(d->ab_ptrs);
+    cudaFree(d->c_ptrs); cudaFree(d->ldcs); cudaFree(d->fin_ref0); cudaFree(d->fin_refs); cudaFree(d->fin_count);
+    cudaFree(d->level_left); cudaFree(d->gemm_table); cudaFree(d->ksplit_table); cudaFree(d->ab_ptrs);
     cudaFree(d->verify_out);
     for (auto& e : d->ev) if (e) cudaEventDestroy(e);
     cudaGetLastError();
@@ -258,14 +293,26 @@ void device_state_free(DeviceState* d) {
 
 }  // namespace cleave
 
+// Checks cleave_assemble_static shares with cleave_assemble (the plan's device state is private to this file).
+int cleave::static_assemble_check(const cleave_plan_s* p, float* const* C) {
+    if (!p->dev) return 0;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CLEAVE_E_CUDA; }
+    if (dev != p->dev->device) return CLEAVE_E_INVAL;          // the plan's blocks live on another device
+    const size_t n = p->gemms.size();
+    void* const* Cv = reinterpret_cast<void* const*>(C);
+    if ((p->fused || p->finished) && (p->dev->last_c.size() != n || !std::equal(Cv, Cv + n, p->dev->last_c.begin())))
+        return CLEAVE_E_INVAL;                                   // part of the result sits in the C the execution was given
+    return 0;
+}
+
 using namespace cleave;
 
 extern "C" {
 
 void cleave_plan_opts_default(cleave_plan_opts_t* o) {
     if (!o) return;
-    o->gran_m = 256;            // rows of an exec-kernel tile: blocks of whole tiles waste no MMA work
-    o->gran_n = o->gran_k = 128;
+    o->gran_m = o->gran_n = o->gran_k = 128;
     o->kslice_max = 4096;
     o->ksplit = 0;
     o->ksplit_cap = 8;
@@ -318,11 +365,23 @@ uint32_t cleave_plan_ksplit(const cleave_plan_t* p, uint32_t gemm) { return (p &
 uint64_t cleave_plan_makespan_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->makespan.size()) ? p->makespan[gemm] : 0; }
 uint64_t cleave_plan_tstar_ns(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->tstar.size()) ? p->tstar[gemm] : 0; }
 uint32_t cleave_plan_num_tiles(const cleave_plan_t* p) { return p ? (uint32_t)p->tiles.size() : 0; }
+uint32_t cleave_plan_finishable(const cleave_plan_t* p, uint32_t gemm) { return (p && gemm < p->gemm_finishable.size()) ? p->gemm_finishable[gemm] : 0; }
+uint32_t cleave_plan_num_levels(const cleave_plan_t* p) { return p ? p->n_levels : 0; }
+uint64_t cleave_plan_level_makespan_ns(const cleave_plan_t* p, uint32_t level) {
+    uint64_t worst = 0;
+    if (p) for (size_t g = 0; g < p->gemms.size(); ++g) if (p->gemms[g].level == level) worst = std::max(worst, p->makespan[g]);
+    return worst;
+}
+uint64_t cleave_plan_step_makespan_ns(const cleave_plan_t* p) {
+    uint64_t sum = 0;
+    if (p) for (uint32_t l = 0; l < p->n_levels; ++l) sum += cleave_plan_level_makespan_ns(p, l);
+    return sum;
+}
 
 uint32_t cleave_plan_num_launches(const cleave_plan_t* p) {
     if (!p) return 0;
     uint32_t n = 5;          // clear + arm + exec, clear verdict + bookkeeping check, then the assembly kernels
-    for (const auto& grp : p->asm_groups) if (!(p->fused && grp.single)) ++n;
+    for (const auto& grp : p->asm_groups) if (!((p->fused && grp.single) || (p->finished && grp.finishable))) ++n;
     return n;
 }
 uint32_t cleave_task_num_tiles(const cleave_plan_t* p, uint32_t task) { return (p && task < p->task_ntiles.size()) ? p->task_ntiles[task] : 0; }
@@ -336,31 +395,46 @@ int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t n) {
     return 0;
 }
 
-int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials, void* stream) {
+int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials, void* const* C,
+                     uint32_t flags, uint32_t level_begin, uint32_t level_end, void* stream) {
     int rc = check_exec_args(p, A, B, partials);
     if (rc) return rc;
+    if (flags & ~(uint32_t)(CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH | CLEAVE_EXEC_BF16)) return CLEAVE_E_INVAL;
+    if ((flags & (CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH)) && !C) return CLEAVE_E_INVAL;
+    if (level_begin > level_end) return CLEAVE_E_INVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     try {
         RC_TRY(sync_device_state(p, st));
         RC_TRY(update_maps(p, A, B, st));
+        if (C) RC_TRY(upload_c_ptrs(p, C, st));
     } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
-    p->fused = false;
-    return run_tiles(p, 0, (uint32_t)p->tiles.size(), 0, (uint32_t)p->tasks.size(), 1, partials, st);
+    p->mode = ((flags & CLEAVE_EXEC_DIRECT) ? MODE_DIRECT : 0u) | ((flags & CLEAVE_EXEC_FINISH) ? MODE_FINISH : 0u) |
+              ((flags & CLEAVE_EXEC_BF16) ? MODE_BF16 : 0u);
+    p->fused = (p->mode & MODE_DIRECT) != 0;
+    p->out_bf16 = (p->mode & MODE_BF16) != 0;
+    // the exec kernel sums every cell of the finishable GEMMs itself unless a block is going to be missing
+    bool whole = level_begin == 0 && level_end >= p->n_levels;
+    for (size_t i = 0; whole && i < p->tasks.size(); ++i)
+        if (p->dropped[i] || (p->tasks[i].flags & CLEAVE_TASK_SUPERSEDED)) whole = false;   // replacement pieces join no cell
+    p->finished = (p->mode & MODE_FINISH) && whole;
+    return run_tiles(p, 0, (uint32_t)p->tiles.size(), true, level_begin, level_end, partials, st);
+}
+
+int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials, void* stream) {
+    return cleave_exec_opts(p, A, B, partials, nullptr, 0u, 0u, 0xFFFFFFFFu, stream);
 }
 
 int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials, float* const* C,
                       void* stream) {
-    int rc = check_exec_args(p, A, B, partials);
-    if (rc) return rc;
     if (!C) return CLEAVE_E_INVAL;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    try {
-        RC_TRY(sync_device_state(p, st));
-        RC_TRY(update_maps(p, A, B, st));
-        RC_TRY(upload_c_ptrs(p, C, st));
-    } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
-    p->fused = true;
-    return run_tiles(p, 0, (uint32_t)p->tiles.size(), 0, (uint32_t)p->tasks.size(), 1, partials, st);
+    return cleave_exec_opts(p, A, B, partials, reinterpret_cast<void* const*>(C), CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH, 0u,
+                            0xFFFFFFFFu, stream);
+}
+
+int cleave_set_wait_limit_ns(cleave_plan_t* p, uint64_t ns) {
+    if (!p) return CLEAVE_E_INVAL;
+    p->wait_limit_ns = ns;
+    return 0;
 }
 
 int cleave_assemble(cleave_plan_t* p, const float* partials, float* const* C, void* stream) {
@@ -370,14 +444,18 @@ int cleave_assemble(cleave_plan_t* p, const float* partials, float* const* C, vo
     try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     DeviceState* d = p->dev;
     const size_t n = p->gemms.size();
+    void* const* Cv = reinterpret_cast<void* const*>(C);
     // after a fused execution part of the result already sits in the C it was given: it must be the same C
-    if (p->fused && (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin()))) return CLEAVE_E_INVAL;
-    try { RC_TRY(upload_c_ptrs(p, C, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    if ((p->fused || p->finished) && (d->last_c.size() != n || !std::equal(Cv, Cv + n, d->last_c.begin()))) return CLEAVE_E_INVAL;
+    try { RC_TRY(upload_c_ptrs(p, Cv, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     CU_TRY(launch_check_done(d->tasks, d->done, d->ntiles, d->tasks_n, d->words + 1, st));
     CU_TRY(cudaEventRecord(d->ev[2], st));
-    for (const auto& grp : p->asm_groups)
-        if (!(p->fused && grp.single))            // one-slice blocks were written to C by the exec kernel
-        CU_TRY(launch_assemble(d->asm_items, d->asm_refs, grp.item0, grp.n_items, grp.sp, partials, d->c_ptrs, d->ldcs, st));
+    for (const auto& grp : p->asm_groups) {
+        // blocks of one-slice GEMMs were written to C, cells of finishable GEMMs summed, by the exec kernel
+        if ((p->fused && grp.single) || (p->finished && grp.finishable)) continue;
+        CU_TRY(launch_assemble(d->asm_items, d->asm_refs, grp.item0, grp.n_items, grp.sp, partials, d->c_ptrs, d->ldcs,
+                               p->out_bf16 ? 1 : 0, st));
+    }
     CU_TRY(cudaEventRecord(d->ev[3], st));
     d->ev_asm = true;
     return 0;
@@ -412,7 +490,16 @@ int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t n, const v
         if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
         RC_TRY(sync_device_state(p, st));
         RC_TRY(update_maps(p, A, B, st));
-        return run_tiles(p, tiles_before, (uint32_t)p->tiles.size(), first_new, (uint32_t)p->tasks.size(), 0, partials, st);
+        p->finished = false;                           // cells that lost a block are summed by cleave_assemble
+        rc = run_tiles(p, tiles_before, (uint32_t)p->tiles.size(), false, 0u, 0xFFFFFFFFu, partials, st);
+        if (p->n_levels > 1) {
+            // the scheduler takes levels in list order: keep the whole list sorted by level for later executions
+            std::stable_sort(p->tiles.begin(), p->tiles.end(), [](const TileDesc& x, const TileDesc& y) {
+                return (x.level & 0xFFFFu) < (y.level & 0xFFFFu);
+            });
+            p->dev->tiles_dirty = true;
+        }
+        return rc;
     } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
 }
 
@@ -426,6 +513,7 @@ int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, 
     if (!p || !A || !B || !partials || !n_bad || !(tol >= 0.f)) return CLEAVE_E_INVAL;
     for (const auto& g : p->gemms) if ((g.K % 4) || (g.lda % 8) || (g.ldb % 8)) return CLEAVE_E_UNSUPPORTED;
     if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
+    if (p->fused && p->out_bf16) return CLEAVE_E_UNSUPPORTED;      // blocks written to C as bf16 are not checked
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     DeviceState* d = p->dev;
@@ -453,7 +541,7 @@ int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, 
     if (sign_bytes > 200 * 1024) return CLEAVE_E_UNSUPPORTED;
     CU_TRY(cudaMemcpyAsync(d->ab_ptrs, ab.data(), ab.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
     CU_TRY(cudaMemsetAsync(d->words + 3, 0, sizeof(unsigned int), st));
-    CU_TRY(launch_verify(d->tasks, d->tasks_n, d->gemm_table, d->ksplit_table, d->ab_ptrs, partials, d->c_ptrs, p->fused ? 1 : 0,
+    CU_TRY(launch_verify(d->tasks, d->tasks_n, d->gemm_table, d->ksplit_table, d->ab_ptrs, partials, reinterpret_cast<float* const*>(d->c_ptrs), p->fused ? 1 : 0,
                          seed, tol, d->verify_out, d->words + 3, sign_bytes, st));
     d->verify_n = d->tasks_n;
     unsigned int bad = 0;

@@ -1,13 +1,15 @@
 // CUDA kernels of the Cleave hot path for sm_100a.
 //
-//   arm_queue_kernel    marks each work-list tile runnable or skipped (dropped / superseded task),
-//                       clears the bookkeeping of the tasks about to run, resets the ticket
+//   arm_queue_kernel    marks each half of every work-list entry runnable or skipped (dropped /
+//                       superseded task), clears the bookkeeping of the tasks about to run, counts
+//                       the strips each DAG level has to finish, resets the ticket
 //   (the grouped GEMM itself, exec_pair_kernel, lives in kernels_pair.cu)
 //   check_done_kernel   flags E_INCOMPLETE if a live task has unfinished tiles
 //   assemble_kernel     fixed-order sum of the K-slices' partial blocks into C
 //   collect_failed_kernel  lists the live tasks whose bookkeeping shows unfinished tiles
 //
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -22,29 +24,33 @@ __global__ void clear_status_bits_kernel(unsigned int* status, unsigned int mask
 // -------------------------------------------------------------------------------------------------
 // arm_queue_kernel
 // -------------------------------------------------------------------------------------------------
-__global__ void arm_queue_kernel(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
-                                 const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                                 unsigned int* ticket, unsigned int* status, int direct, unsigned long long arena_elems) {
+__global__ void arm_queue_kernel(const ArmParams a) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i == 0) {
-        *ticket = tile_begin;
-    }
-    const uint32_t t = tile_begin + i;
-    if (t < tile_end) {
-        const uint32_t task = tiles[t].task;
-        const bool skip = dropped[task] || (tasks[task].flags & CLEAVE_TASK_SUPERSEDED);
-        uint32_t f = tiles[t].flags & ~(uint32_t)(TILE_VALID | TILE_DIRECT);
-        if (!skip) f |= TILE_VALID;
-        if (direct && (f & TILE_SINGLE)) f |= TILE_DIRECT;
-        // range check of the block the tile will write: a tile that would leave the arena is not run
-        if (!(f & TILE_DIRECT) && tiles[t].out_off + (unsigned long long)(tiles[t].rows - 1) * tiles[t].ld + tiles[t].cols > arena_elems) {
-            f &= ~(uint32_t)TILE_VALID;
-            atomicOr(status, STATUS_BOUNDS);
+    if (i == 0) *a.ticket = a.tile_begin;
+    const uint32_t t = a.tile_begin + i;
+    if (t >= a.tile_end) return;
+    TileDesc& d = a.tiles[t];
+    uint32_t f = d.flags & ~(uint32_t)(TILE_LIVE0 | TILE_LIVE1);
+    const bool direct = (a.mode & MODE_DIRECT) && (f & TILE_SINGLE);
+    const uint32_t cols = d.n_mma >> 16;
+    uint32_t live = 0;
+    const uint32_t level = d.level & 0xFFFFu;
+    const bool in_range = level >= a.level_begin && level < a.level_end;
+    for (uint32_t r = 0; r < 2; ++r) {
+        const TileHalf& h = d.h[r];
+        if (h.rows == 0 || !in_range) continue;
+        a.done[h.task] = 0;                              // every tile of the task writes the same value
+        if (a.dropped[h.task] || (a.tasks[h.task].flags & CLEAVE_TASK_SUPERSEDED)) continue;
+        // range check of the block the half-tile will write: one that would leave the arena is not run
+        if (!direct && h.out_off + (unsigned long long)(h.rows - 1) * h.ld + cols > a.arena_elems) {
+            atomicOr(a.status, STATUS_BOUNDS);
+            continue;
         }
-        tiles[t].flags = f;
+        f |= TILE_LIVE0 << r;
+        ++live;
     }
-    const uint32_t k = task_begin + i;
-    if (k < task_end) done[k] = 0;
+    d.flags = f;
+    if (live) atomicAdd(&a.level_left[level], live * (uint32_t)kEpiWarpsPerGroup);
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -78,11 +84,15 @@ __global__ void collect_failed_kernel(const cleave_task_t* tasks, const uint32_t
 // each lane sums its R slices as a balanced tree in registers, then a butterfly of shfl_xor over the
 // group index finishes the balanced tree over all SP slices.  Either way the order is the fixed
 // balanced pairwise tree over adjacent slices, so the sum is deterministic; missing slices
-// (s >= nslices) contribute +0.0f.
-template <int SP>
+// (s >= nslices) contribute +0.0f.  BF16: C holds bf16, each sum is rounded to nearest even.
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+template <int SP, bool BF16>
 __global__ void __launch_bounds__(256)
 assemble_vec_kernel(const AsmItem* __restrict__ items, const AsmRef* __restrict__ refs, uint32_t item0,
-                    const float* __restrict__ partials, float* const* __restrict__ Cptr, const uint32_t* __restrict__ ldcs) {
+                    const float* __restrict__ partials, void* const* __restrict__ Cptr, const uint32_t* __restrict__ ldcs) {
     constexpr int G = SP <= 4 ? 1 : 8;
     constexpr int R = SP / G;
     constexpr int LG = 32 / G;
@@ -102,7 +112,9 @@ assemble_vec_kernel(const AsmItem* __restrict__ items, const AsmRef* __restrict_
         if (s < it.nslices) { const AsmRef rf = refs[it.ref0 + s]; src[r] = partials + rf.off; ld[r] = rf.ld; }
         else { src[r] = nullptr; ld[r] = 0; }
     }
-    float* crow = Cptr[it.gemm] + (uint64_t)it.i0 * ldc + it.j0;
+    const uint64_t c_at = (uint64_t)it.i0 * ldc + it.j0;
+    float* crow = static_cast<float*>(Cptr[it.gemm]) + c_at;
+    __nv_bfloat16* crow16 = static_cast<__nv_bfloat16*>(Cptr[it.gemm]) + c_at;
 
     for (uint32_t base = warp * (LG * U); base < units; base += nwarps * (LG * U)) {
         float4 acc[U];
@@ -139,19 +151,23 @@ assemble_vec_kernel(const AsmItem* __restrict__ items, const AsmRef* __restrict_
         if (g == 0) {
 #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (base + u * LG + l < units)
-                    __stcs(reinterpret_cast<float4*>(crow + (uint64_t)urow[u] * ldc + ucol[u]), acc[u]);
+                if (base + u * LG + l < units) {
+                    if (BF16) __stcs(reinterpret_cast<uint2*>(crow16 + (uint64_t)urow[u] * ldc + ucol[u]),
+                                     make_uint2(pack2_bf16(acc[u].x, acc[u].y), pack2_bf16(acc[u].z, acc[u].w)));
+                    else      __stcs(reinterpret_cast<float4*>(crow + (uint64_t)urow[u] * ldc + ucol[u]), acc[u]);
+                }
         }
     }
 }
 
 // Any alignment, any slice count up to 32: one thread per output element, the same balanced tree.
 __global__ void assemble_scalar_kernel(const AsmItem* __restrict__ items, const AsmRef* __restrict__ refs, uint32_t item0,
-                                       const float* __restrict__ partials, float* const* __restrict__ Cptr,
-                                       const uint32_t* __restrict__ ldcs) {
+                                       const float* __restrict__ partials, void* const* __restrict__ Cptr,
+                                       const uint32_t* __restrict__ ldcs, int out_bf16) {
     const AsmItem it = items[item0 + blockIdx.x];
     const uint32_t ldc = ldcs[it.gemm];
-    float* C = Cptr[it.gemm];
+    float* C = static_cast<float*>(Cptr[it.gemm]);
+    __nv_bfloat16* C16 = static_cast<__nv_bfloat16*>(Cptr[it.gemm]);
     uint32_t sp = 1;
     while (sp < it.nslices) sp *= 2;
     const uint32_t n = it.nrows * it.ncols;
@@ -164,24 +180,20 @@ __global__ void assemble_scalar_kernel(const AsmItem* __restrict__ items, const 
         }
         for (uint32_t w = 1; w < sp; w *= 2)
             for (uint32_t s = 0; s < sp; s += 2 * w) v[s] += v[s + w];
-        C[(uint64_t)(it.i0 + r) * ldc + it.j0 + c] = v[0];
+        if (out_bf16) C16[(uint64_t)(it.i0 + r) * ldc + it.j0 + c] = __float2bfloat16_rn(v[0]);
+        else          C[(uint64_t)(it.i0 + r) * ldc + it.j0 + c] = v[0];
     }
 }
 
 // -------------------------------------------------------------------------------------------------
 // host-side launchers
 // -------------------------------------------------------------------------------------------------
-cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
-                             const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, uint64_t arena_elems,
-                             cudaStream_t st) {
-    uint32_t n = tile_end - tile_begin;
-    if (task_end - task_begin > n) n = task_end - task_begin;
+cudaError_t launch_arm_queue(const ArmParams& a, int clear_status, cudaStream_t st) {
+    uint32_t n = a.tile_end - a.tile_begin;
     if (n == 0) n = 1;
     // a fresh execution forgets the verdicts of the previous one (before the arming threads may raise new ones)
-    if (clear_status) clear_status_bits_kernel<<<1, 1, 0, st>>>(status, 0xFFFFFFFFu);
-    arm_queue_kernel<<<(n + 255) / 256, 256, 0, st>>>(tiles, tile_begin, tile_end, tasks, dropped, done, task_begin,
-                                                       task_end, ticket, status, direct, (unsigned long long)arena_elems);
+    if (clear_status) clear_status_bits_kernel<<<1, 1, 0, st>>>(a.status, 0xFFFFFFFFu);
+    arm_queue_kernel<<<(n + 255) / 256, 256, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -201,20 +213,30 @@ cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* do
     return cudaGetLastError();
 }
 
-cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
-                            const float* partials, float* const* Cptr, const uint32_t* ldcs, cudaStream_t st) {
-    if (!n_items) return cudaSuccess;
+template <bool BF16>
+static cudaError_t launch_assemble_vec(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
+                                       const float* partials, void* const* Cptr, const uint32_t* ldcs, cudaStream_t st) {
     switch (sp) {
-        case 0:  assemble_scalar_kernel<<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
-        case 1:  assemble_vec_kernel<1><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
-        case 2:  assemble_vec_kernel<2><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
-        case 4:  assemble_vec_kernel<4><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
-        case 8:  assemble_vec_kernel<8><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
-        case 16: assemble_vec_kernel<16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
-        case 32: assemble_vec_kernel<32><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 1:  assemble_vec_kernel<1, BF16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 2:  assemble_vec_kernel<2, BF16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 4:  assemble_vec_kernel<4, BF16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 8:  assemble_vec_kernel<8, BF16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 16: assemble_vec_kernel<16, BF16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
+        case 32: assemble_vec_kernel<32, BF16><<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
+}
+
+cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
+                            const float* partials, void* const* Cptr, const uint32_t* ldcs, int out_bf16, cudaStream_t st) {
+    if (!n_items) return cudaSuccess;
+    if (sp == 0) {
+        assemble_scalar_kernel<<<n_items, 256, 0, st>>>(items, refs, item0, partials, Cptr, ldcs, out_bf16);
+        return cudaGetLastError();
+    }
+    return out_bf16 ? launch_assemble_vec<true>(items, refs, item0, n_items, sp, partials, Cptr, ldcs, st)
+                    : launch_assemble_vec<false>(items, refs, item0, n_items, sp, partials, Cptr, ldcs, st);
 }
 
 }  // namespace cleave
@@ -254,6 +276,8 @@ extern "C" int cleave_assemble_static(cleave_plan_t* p, const float* partials, f
     for (uint32_t s : p->ksplit) if (s > 32) return CLEAVE_E_UNSUPPORTED;
     const size_t n = p->gemms.size();
     for (size_t i = 0; i < n; ++i) if (!C[i] || ((uintptr_t)C[i] & 15)) return CLEAVE_E_INVAL;
+    const int chk = cleave::static_assemble_check(p, C);
+    if (chk) return chk;
     // layout of the fixed array: items | refs | output pointers | leading dimensions
     const size_t items_b = p->asm_items.size() * sizeof(cleave::AsmItem), refs_b = p->asm_refs.size() * sizeof(cleave::AsmRef);
     const size_t off_refs = round256(items_b), off_ptrs = off_refs + round256(refs_b), off_ld = off_ptrs + round256(n * sizeof(float*));
@@ -274,10 +298,10 @@ extern "C" int cleave_assemble_static(cleave_plan_t* p, const float* partials, f
         return CLEAVE_E_CUDA;
     }
     for (const auto& grp : p->asm_groups) {
-        if (p->fused && grp.single) continue;         // those blocks were written to C by the exec kernel
+        if ((p->fused && grp.single) || (p->finished && grp.finishable)) continue;   // already in C, written by the exec kernel
         if (cleave::launch_assemble(reinterpret_cast<const cleave::AsmItem*>(base), reinterpret_cast<const cleave::AsmRef*>(base + off_refs),
-                                    grp.item0, grp.n_items, grp.sp, partials, reinterpret_cast<float* const*>(base + off_ptrs),
-                                    reinterpret_cast<const uint32_t*>(base + off_ld), st) != cudaSuccess) {
+                                    grp.item0, grp.n_items, grp.sp, partials, reinterpret_cast<void* const*>(base + off_ptrs),
+                                    reinterpret_cast<const uint32_t*>(base + off_ld), p->out_bf16 ? 1 : 0, st) != cudaSuccess) {
             cudaGetLastError();
             return CLEAVE_E_CUDA;
         }

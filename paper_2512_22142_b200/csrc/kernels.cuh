@@ -23,6 +23,7 @@ constexpr int kAccSlots = 2;                         // accumulator slots in ten
 constexpr uint32_t kAccCols = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSchedSlots = 4;
+constexpr int kTileWords16 = sizeof(TileDesc) / 16;   // 16-byte words of a work-list entry
 constexpr uint32_t kEpiStageFloats = 32 * 33;        // per epilogue warp: padded 32 x 32 transpose tile
 
 constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4;
@@ -30,19 +31,45 @@ constexpr int kEpiWarpsPerGroup = 4, kEpiWarps = 2 * kEpiWarpsPerGroup;   // gro
 constexpr int kExecThreads = 32 * (kEpiWarp0 + kEpiWarps);
 constexpr uint32_t kPairDynSmem = kPairStages * kPairStageBytes + 1024 + kEpiWarps * kEpiStageFloats * 4;
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;     // bound of every device-side wait
-
 // device status word bits
 enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BOUNDS = 2u, STATUS_INCOMPLETE = 4u };
 
-cudaError_t launch_arm_queue(TileDesc* tiles, uint32_t tile_begin, uint32_t tile_end, const cleave_task_t* tasks,
-                             const uint8_t* dropped, uint32_t* done, uint32_t task_begin, uint32_t task_end,
-                             unsigned int* ticket, unsigned int* status, int clear_status, int direct, uint64_t arena_elems,
-                             cudaStream_t st);
+// Arguments of the exec kernel (passed by value).
+struct ExecParams {
+    const TileDesc* tiles;          // work list (device)
+    uint32_t tile_end;              // the ticket runs up to here
+    unsigned int* ticket;
+    const CUtensorMap* maps;        // kMapsPerGemm per GEMM
+    float* partials;                // arena
+    void* const* c_ptrs;            // per GEMM: C (fp32, or bf16 under MODE_BF16)
+    uint32_t* done;                 // per task: finished half-tiles x epilogue warps
+    unsigned int* status;
+    const uint32_t* fin_ref0;       // per cell: first entry in fin_refs
+    const FinRef* fin_refs;
+    unsigned int* fin_count;        // per cell and 32-row strip: blocks arrived
+    unsigned int* level_left;       // per DAG level: epilogue-warp strips still to finish
+    uint32_t mode;                  // MODE_*
+    unsigned long long wait_limit_ns;   // bound of every device-side wait
+};
+
+// Words of a launch's arming kernel.
+struct ArmParams {
+    TileDesc* tiles;
+    uint32_t tile_begin, tile_end;
+    const cleave_task_t* tasks;
+    const uint8_t* dropped;
+    uint32_t* done;
+    unsigned int* ticket;
+    unsigned int* status;
+    unsigned int* level_left;
+    uint32_t mode;
+    uint32_t level_begin, level_end;   // only tiles of these DAG levels run
+    unsigned long long arena_elems;
+};
+
+cudaError_t launch_arm_queue(const ArmParams& a, int clear_status, cudaStream_t st);
 cudaError_t exec_pair_kernel_prepare();
-cudaError_t launch_exec_pair(uint32_t clusters, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
-                             const CUtensorMap* maps, float* partials, float* const* c_ptrs, uint32_t* done,
-                             unsigned int* status, cudaStream_t st);
+cudaError_t launch_exec_pair(uint32_t clusters, const ExecParams& e, cudaStream_t st);
 cudaError_t launch_check_done(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles, uint32_t n_tasks,
                               unsigned int* status, cudaStream_t st);
 cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* done, const uint32_t* ntiles,
@@ -50,8 +77,8 @@ cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* do
 cudaError_t launch_verify(const cleave_task_t* tasks, uint32_t n_tasks, const cleave_gemm_t* gemms, const uint32_t* ksplit,
                           const void* const* ab_ptrs, const float* partials, float* const* c_ptrs, int fused, uint64_t seed,
                           float tol, float4* out, unsigned int* n_bad, uint32_t sign_bytes, cudaStream_t st);
-// sp = padded slice count of the vectorised kernel (1, 2, 4, 8, 16, 32), 0 = scalar kernel
+// sp = padded slice count of the vectorised kernel (1, 2, 4, 8, 16, 32), 0 = scalar kernel; out_bf16: C holds bf16
 cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
-                            const float* partials, float* const* Cptr, const uint32_t* ldcs, cudaStream_t st);
+                            const float* partials, void* const* Cptr, const uint32_t* ldcs, int out_bf16, cudaStream_t st);
 
 }  // namespace cleave

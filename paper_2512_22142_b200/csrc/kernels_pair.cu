@@ -1,13 +1,14 @@
 // exec_pair_kernel: the grouped sub-GEMM kernel on pairs of CTAs (thread-block clusters of two,
 // tcgen05 cta_group::2).
 //
-// A tile of up to 256 rows x up to 256 columns is shared by the two CTAs of a cluster: CTA r loads
-// rows 128r..128r+127 of A and columns r*N/2..(r+1)*N/2-1 of B into its own shared memory, one
-// thread of the leader CTA (rank 0) issues M = 256 MMAs that read both CTAs' shared memory, and each
-// CTA receives its 128 rows of the accumulator in its own tensor memory.  Compared with one CTA
-// doing both row halves this halves, per SM, the B bytes held, loaded and read by the tensor core
-// and the accumulator columns, so six 32 KB stages fit and two accumulator slots double-buffer:
-// the write-out of a tile overlaps the MMAs of the next one.
+// The unit of work is a pair of half-tiles (up to 128 rows x up to 256 columns each, same GEMM, K-range
+// and columns) shared by the two CTAs of a cluster: CTA r loads the rows of half r of A and columns
+// r*N/2..(r+1)*N/2-1 of B into its own shared memory, one thread of the leader CTA (rank 0) issues
+// M = 256 MMAs that read both CTAs' shared memory, and each CTA receives the 128 accumulator rows of
+// its half in its own tensor memory and writes them out.  The halves may lie anywhere in the GEMM and
+// belong to different tasks.  Compared with one CTA doing both row halves this halves, per SM, the B
+// bytes held, loaded and read by the tensor core and the accumulator columns, so six 32 KB stages
+// fit and two accumulator slots double-buffer: the write-out of a tile overlaps the MMAs of the next.
 //
 // Synchronisation between the two CTAs uses only mbarriers:
 //   full[s]      leader's barrier; the leader's producer arms it with the bytes of BOTH CTAs, and
@@ -21,11 +22,25 @@
 // Every TMA load is an ordinary load into the issuing CTA's own shared memory (no load is shared
 // between CTAs).
 //
+// Write-out (epilogue warps, each owning a strip of 32 accumulator rows).  The strip always goes to
+// the task's packed block in the arena, or, for a GEMM with one K-slice under MODE_DIRECT, to its
+// place in C.  Under MODE_FINISH a strip of a GEMM with several K-slices then counts its arrival at
+// its cell; the strip that arrives last reads the cell's blocks of all K-slices back (they are in
+// L2: the slices of a cell follow each other in the work list), sums them in the fixed balanced-tree
+// order -- the order does not depend on which block arrived last -- and writes C.  Under MODE_BF16
+// values written to C are rounded to bf16.
+//
+// DAG levels: tiles are ordered by level, and before the scheduler hands out the first tile of a
+// level it waits until every strip of the lower levels has been written (a counter per level that
+// the epilogue warps count down after their stores), so a GEMM may read what a GEMM of a lower
+// level wrote in the same launch.
+//
 // Every device-side wait is bounded: when a wait expires the CTA records E_TIMEOUT in the status
-// word and raises its abort flag, all its roles leave their loops, the MMAs in flight are drained
-// (again with a bound), both CTAs meet at the cluster barrier, tensor memory is released and the
-// kernel returns.
+// word and raises the abort flag of both CTAs, all roles leave their loops, the MMAs in flight are
+// drained (again with a bound), both CTAs meet at the cluster barrier, tensor memory is released
+// and the kernel returns.
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -63,29 +78,48 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cl(uint32_t bar, uint32_t pari
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
-static __device__ __noinline__ bool mbar_wait_cl_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                               unsigned int* status) {
+// What every wait of this kernel needs to know to give up.
+struct WaitCtx {
+    volatile uint32_t* abort_flag;
+    unsigned int* status;
+    uint64_t limit_ns;
+};
+// Both CTAs of the pair give up: every role leaves at its next check.
+__device__ __forceinline__ void raise_abort(const WaitCtx& w) {
+    const uint32_t flag = smem_u32(const_cast<uint32_t*>(w.abort_flag));
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(flag, 0u)), "r"(1u) : "memory");
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(flag, 1u)), "r"(1u) : "memory");
+    atomicOr(w.status, STATUS_TIMEOUT);
+}
+static __device__ __noinline__ bool mbar_wait_cl_slow(uint32_t bar, uint32_t parity, const WaitCtx& w) {
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait_cl(bar, parity)) {
-        if ((++spins & 255u) == 0) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
-                // give up: raise the abort flag of both CTAs of the pair so that every role leaves at its next check
-                const uint32_t flag = smem_u32(const_cast<uint32_t*>(abort_flag));
-                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(flag, 0u)), "r"(1u) : "memory");
-                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(flag, 1u)), "r"(1u) : "memory");
-                atomicOr(status, STATUS_TIMEOUT);
-                return false;
-            }
+        if ((spins++ & 255u) == 0) {                     // at the first unsuccessful poll, then every 256
+            if (*w.abort_flag) return false;
+            if (global_timer_ns() - t0 >= w.limit_ns) { raise_abort(w); return false; }
         }
     }
     return true;
 }
-__device__ __forceinline__ bool mbar_wait_cl(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                             unsigned int* status) {
+__device__ __forceinline__ bool mbar_wait_cl(uint32_t bar, uint32_t parity, const WaitCtx& w) {
     if (mbar_try_wait_cl(bar, parity)) return true;
-    return mbar_wait_cl_slow(bar, parity, abort_flag, status);
+    return mbar_wait_cl_slow(bar, parity, w);
+}
+// Bounded wait for a counter in global memory to reach zero (written by other clusters' epilogue warps).
+static __device__ __noinline__ bool wait_zero(const unsigned int* ctr, const WaitCtx& w) {
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    for (;;) {
+        unsigned int v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v == 0) return true;
+        if ((spins++ & 63u) == 0) {
+            if (*w.abort_flag) return false;
+            if (global_timer_ns() - t0 >= w.limit_ns) { raise_abort(w); return false; }
+        }
+        __nanosleep(64);
+    }
 }
 __device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint4 v) {
     asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -123,19 +157,23 @@ __device__ __forceinline__ void umma_commit_both(uint32_t bar) {
 __device__ __forceinline__ void umma_commit_local_pair(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-
-// rows of the tile that belong to CTA `rank` (0..128)
-__device__ __forceinline__ uint32_t rows_of_rank(uint32_t tile_rows, uint32_t rank) {
-    const uint32_t lo = rank * kBlockM;
-    return tile_rows > lo ? min(kBlockM, tile_rows - lo) : 0u;
+// loads that must see what other SMs wrote a moment ago: from L2, never from this SM's L1
+__device__ __forceinline__ float4 ld_cg_f4(const float* p) {
+    float4 v;
+    asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
 }
-// bytes CTA `rank` loads per K-block of tile d
-__device__ __forceinline__ uint32_t stage_bytes_of_rank(uint32_t tile_rows, uint32_t n_mma, uint32_t rank) {
-    const uint32_t nsub_a = (rows_of_rank(tile_rows, rank) + kSubRows - 1) / kSubRows;
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);      // round to nearest even; .x = lo is the low half
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// bytes CTA with `rows` valid rows loads per K-block of a pair whose MMA is n_mma columns wide
+__device__ __forceinline__ uint32_t stage_bytes(uint32_t rows, uint32_t n_mma) {
+    const uint32_t nsub_a = (rows + kSubRows - 1) / kSubRows;
     const uint32_t nsub_b = (n_mma / 2 + kSubRows - 1) / kSubRows;
     return (nsub_a + nsub_b) * kSubBytes;
 }
-
 struct __align__(16) PairShared {
     uint64_t full[kPairStages];
     uint64_t empty[kPairStages];
@@ -149,17 +187,65 @@ struct __align__(16) PairShared {
     TileDesc slot[kSchedSlots];
 };
 
+// Sum of the SP (slice count padded to a power of two) blocks of a cell for one 32-row strip, in
+// the order of the assembly kernel: balanced pairwise tree over adjacent slices, missing slices
+// contribute +0.0f.  One float4 per lane and step, four steps in flight.
+template <int SP, bool BF16>
+__device__ __forceinline__ void finish_strip(const FinRef* __restrict__ refs, uint32_t nslices, const float* __restrict__ partials,
+                                             uint32_t row0, uint32_t nrows, uint32_t cols, void* c_base, uint64_t c_off,
+                                             uint32_t ldc, uint32_t lane) {
+    constexpr int U = 4;
+    const float* src[SP];
+    uint32_t ld[SP];
+#pragma unroll
+    for (int s = 0; s < SP; ++s) {
+        if ((uint32_t)s < nslices) { const FinRef rf = refs[s]; src[s] = partials + rf.off + (uint64_t)row0 * rf.ld; ld[s] = rf.ld; }
+        else { src[s] = nullptr; ld[s] = 0; }
+    }
+    const uint32_t c4 = cols >> 2, units = nrows * c4;
+    for (uint32_t base = 0; base < units; base += 32 * U) {
+        float4 acc[U];
+        uint32_t urow[U], ucol[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t unit = base + u * 32 + lane;
+            const bool live = unit < units;
+            urow[u] = live ? unit / c4 : 0u;
+            ucol[u] = live ? (unit - urow[u] * c4) * 4u : 0u;
+            float4 v[SP];
+#pragma unroll
+            for (int s = 0; s < SP; ++s) {
+                v[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (live && src[s]) v[s] = ld_cg_f4(src[s] + (uint64_t)urow[u] * ld[s] + ucol[u]);
+            }
+#pragma unroll
+            for (int w = 1; w < SP; w *= 2)
+#pragma unroll
+                for (int s = 0; s < SP; s += 2 * w) {
+                    v[s].x += v[s + w].x; v[s].y += v[s + w].y; v[s].z += v[s + w].z; v[s].w += v[s + w].w;
+                }
+            acc[u] = v[0];
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (base + u * 32 + lane >= units) continue;
+            const uint64_t at = c_off + (uint64_t)(row0 + urow[u]) * ldc + ucol[u];
+            if (BF16) *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(c_base) + at) =
+                          make_uint2(pack_bf16(acc[u].x, acc[u].y), pack_bf16(acc[u].z, acc[u].w));
+            else      *reinterpret_cast<float4*>(static_cast<float*>(c_base) + at) = acc[u];
+        }
+    }
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kExecThreads, 1)
-exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned int* ticket,
-                 const CUtensorMap* __restrict__ maps, float* __restrict__ partials, float* const* __restrict__ c_ptrs,
-                 uint32_t* done, unsigned int* status) {
+exec_pair_kernel(const __grid_constant__ ExecParams P) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ PairShared sh;
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
     const uint32_t stage_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
-    volatile uint32_t* abort_flag = &sh.abort_flag;
+    const WaitCtx W = {&sh.abort_flag, P.status, P.wait_limit_ns};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairStages; ++s) { mbar_init(smem_u32(&sh.full[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1); }
@@ -180,24 +266,35 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
     if (warp == kSchedWarp) {
         // ---- scheduler (leader only): ticket -> descriptor -> both CTAs' slot rings -----------------------
         if (rank == 0 && lane == 0) {
+            uint32_t levels_done = 0;                  // every level below this one is known to be complete
             for (uint32_t i = 0;; ++i) {
                 const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-                if (!mbar_wait_cl(smem_u32(&sh.sched_empty[q]), par ^ 1u, abort_flag, status)) break;
-                uint4 w0, w1, w2, w3;
+                if (!mbar_wait_cl(smem_u32(&sh.sched_empty[q]), par ^ 1u, W)) break;
+                uint4 w[kTileWords16];
                 bool end = false;
                 for (;;) {
-                    const uint32_t t = atomicAdd(ticket, 1u);
-                    if (t >= tile_end) { end = true; break; }
-                    const uint4* src = reinterpret_cast<const uint4*>(tiles + t);
-                    w0 = __ldg(src); w1 = __ldg(src + 1); w2 = __ldg(src + 2); w3 = __ldg(src + 3);
-                    if (w0.z & TILE_VALID) break;      // TileDesc::flags
+                    const uint32_t t = atomicAdd(P.ticket, 1u);
+                    if (t >= P.tile_end) { end = true; break; }
+                    const uint4* src = reinterpret_cast<const uint4*>(P.tiles + t);
+#pragma unroll
+                    for (int x = 0; x < kTileWords16; ++x) w[x] = __ldg(src + x);
+                    if (w[0].y & (TILE_LIVE0 | TILE_LIVE1)) break;      // TileDesc::flags
                 }
-                if (end) { w0 = make_uint4(0, 0, TILE_END, 0); w1 = w2 = w3 = make_uint4(0, 0, 0, 0); }
+                if (end) {
+#pragma unroll
+                    for (int x = 0; x < kTileWords16; ++x) w[x] = make_uint4(0, 0, 0, 0);
+                    w[0].y = TILE_END;
+                } else {
+                    // a tile of a higher DAG level runs only after every strip of the lower levels is written
+                    const uint32_t level = w[1].w & 0xFFFFu;         // TileDesc::level
+                    bool ok = true;
+                    while (ok && levels_done < level) { ok = wait_zero(P.level_left + levels_done, W); if (ok) ++levels_done; }
+                    if (!ok) break;
+                }
                 uint4* dst = reinterpret_cast<uint4*>(&sh.slot[q]);
-                dst[0] = w0; dst[1] = w1; dst[2] = w2; dst[3] = w3;
                 const uint32_t peer_slot = mapa_shared(smem_u32(&sh.slot[q]), 1u);
-                st_shared_cluster_v4(peer_slot, w0); st_shared_cluster_v4(peer_slot + 16, w1);
-                st_shared_cluster_v4(peer_slot + 32, w2); st_shared_cluster_v4(peer_slot + 48, w3);
+#pragma unroll
+                for (int x = 0; x < kTileWords16; ++x) { dst[x] = w[x]; st_shared_cluster_v4(peer_slot + 16 * x, w[x]); }
                 mbar_arrive_cluster(mapa_shared(smem_u32(&sh.sched_full[q]), 0u));
                 mbar_arrive_cluster(mapa_shared(smem_u32(&sh.sched_full[q]), 1u));
                 if (end) break;
@@ -205,49 +302,59 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
         }
     } else if (warp == kTmaWarp) {
         // ---- producer (both CTAs): own rows of A, own half of the columns of B ------------------------------
-        uint32_t it = 0, last_gemm = 0xFFFFFFFFu;
+        uint32_t it = 0, last_gemm = 0xFFFFFFFFu, last_level = 0;
         bool ok = true;
         const uint32_t sched_empty_leader0 = mapa_shared(smem_u32(&sh.sched_empty[0]), 0u);
         const uint32_t full_leader0 = mapa_shared(smem_u32(&sh.full[0]), 0u);
         for (uint32_t i = 0; ok; ++i) {
             const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, abort_flag, status))) break;
-            const TileDesc d = sh.slot[q];
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, W))) break;
+            const TileDesc& sl = sh.slot[q];
+            const uint32_t flags = sl.flags, gemm = sl.gemm, level = sl.level & 0xFFFFu, n_mma = sl.n_mma & 0xFFFFu;
+            const uint32_t n_col = sl.n_col, k0 = sl.k0, k1 = sl.k1;
+            const uint32_t rows0 = (flags & TILE_LIVE0) ? sl.h[0].rows : 0u, rows1 = (flags & TILE_LIVE1) ? sl.h[1].rows : 0u;
+            const uint32_t a_x = sl.h[rank].m_row;
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
-            if (d.flags & TILE_END) break;
-            const CUtensorMap* map_a = maps + kMapsPerGemm * d.gemm;
+            if (flags & TILE_END) break;
+            const CUtensorMap* map_a = P.maps + kMapsPerGemm * gemm;
             const CUtensorMap* map_b = map_a + 1;
-            if (d.gemm != last_gemm) {
+            if (gemm != last_gemm) {
                 for (int x = 0; x < kMapsPerGemm; ++x) tensormap_acquire(map_a + x);
-                last_gemm = d.gemm;
+                last_gemm = gemm;
             }
-            const uint32_t half_n = d.n_mma / 2;
-            const uint32_t my_rows = rows_of_rank(d.rows, rank);
-            const uint32_t a_x = d.m_row + rank * kBlockM, b_x = d.n_col + rank * half_n;
+            if (level != last_level) {
+                // operands of this level may have been written by other SMs a moment ago (ordinary stores, seen
+                // through the scheduler's acquire): order them before this thread's asynchronous loads
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                last_level = level;
+            }
+            const uint32_t half_n = n_mma / 2;
+            const uint32_t my_rows = rank ? rows1 : rows0;
+            const uint32_t b_x = n_col + rank * half_n;
             // More than 64 rows / columns of an operand come with ONE operation where a double-size box
             // exists (fewer, larger TMA operations: +9 % on GEMMs whose operands are K-contiguous); an
             // M/N-contiguous operand also needs its first element on a 64-element group boundary.
-            const bool a_big = (d.flags & TILE_A_BIG) && my_rows > kSubRows && (!(d.flags & TILE_A_MN) || a_x % kSubRows == 0);
-            const bool b_big = (d.flags & TILE_B_BIG) && half_n > kSubRows && (!(d.flags & TILE_B_MN) || b_x % kSubRows == 0);
+            const bool a_big = (flags & TILE_A_BIG) && my_rows > kSubRows && (!(flags & TILE_A_MN) || a_x % kSubRows == 0);
+            const bool b_big = (flags & TILE_B_BIG) && half_n > kSubRows && (!(flags & TILE_B_MN) || b_x % kSubRows == 0);
             const uint32_t nsub_a = a_big ? 1u : (my_rows + kSubRows - 1) / kSubRows;
             const uint32_t nsub_b = b_big ? 1u : (half_n + kSubRows - 1) / kSubRows;
             // bytes per stage do not depend on the box size: a double-size box is two 8 KB boxes
-            const uint32_t tx_both = stage_bytes_of_rank(d.rows, d.n_mma, 0u) + stage_bytes_of_rank(d.rows, d.n_mma, 1u);
-            const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
+            const uint32_t tx_both = stage_bytes(rows0, n_mma) + stage_bytes(rows1, n_mma);
+            const uint32_t nkb = (k1 - k0 + kBlockK - 1) / kBlockK;
             const bool is_a = lane < nsub_a, is_b = !is_a && lane < nsub_a + nsub_b;
             const uint32_t j = is_a ? lane : lane - nsub_a;
             const bool my_big = is_a ? a_big : b_big;
             const CUtensorMap* my_map = (is_a ? map_a : map_b) + (my_big ? 2 : 0);
-            const bool my_mn = is_a ? (d.flags & TILE_A_MN) : (d.flags & TILE_B_MN);
+            const bool my_mn = is_a ? (flags & TILE_A_MN) : (flags & TILE_B_MN);
             const int32_t my_x = (int32_t)((is_a ? a_x : b_x) + j * kSubRows);
             const uint32_t my_off = (is_a ? 0u : kPairABytes) + j * kSubBytes;
             for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const uint32_t s = it % kPairStages, ph = (it / kPairStages) & 1u;
-                if (!__all_sync(0xFFFFFFFFu, mbar_wait_cl(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, status))) { ok = false; break; }
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait_cl(smem_u32(&sh.empty[s]), ph ^ 1u, W))) { ok = false; break; }
                 if (rank == 0 && lane == 0) mbar_arrive_expect_tx(smem_u32(&sh.full[s]), tx_both);
                 __syncwarp();
-                const int32_t k = (int32_t)(d.k0 + kb * kBlockK);
+                const int32_t k = (int32_t)(k0 + kb * kBlockK);
                 if (is_a || is_b) {
                     const uint32_t dst = stage_base + s * kPairStageBytes + my_off;
                     const uint32_t bar = full_leader0 + s * 8u;
@@ -260,7 +367,7 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
         // Every stage armed on the normal path has been waited for by the leader's MMA thread, and a stage
         // only completes once this CTA's own bytes have landed.  When the pair is aborting, copies may
         // still be in flight towards this CTA's shared memory: give them a bounded time to land.
-        if (*abort_flag && lane == 0) {
+        if (*W.abort_flag && lane == 0) {
             const uint64_t t0 = global_timer_ns();
             while (global_timer_ns() - t0 < 200000ull) { }
         }
@@ -271,22 +378,23 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
             bool ok = true;
             for (uint32_t i = 0; ok; ++i) {
                 const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-                if (!mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, abort_flag, status)) break;
-                const TileDesc d = sh.slot[q];
+                if (!mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, W)) break;
+                const uint32_t flags = sh.slot[q].flags, n_mma = sh.slot[q].n_mma & 0xFFFFu;
+                const uint32_t k0 = sh.slot[q].k0, k1 = sh.slot[q].k1;
                 mbar_arrive(smem_u32(&sh.sched_empty[q]));
-                if (d.flags & TILE_END) break;
-                const uint32_t a_mn = (d.flags & TILE_A_MN) ? 1u : 0u, b_mn = (d.flags & TILE_B_MN) ? 1u : 0u;
-                const uint32_t idesc = instr_desc_bf16(2 * kBlockM, d.n_mma, a_mn, b_mn);
+                if (flags & TILE_END) break;
+                const uint32_t a_mn = (flags & TILE_A_MN) ? 1u : 0u, b_mn = (flags & TILE_B_MN) ? 1u : 0u;
+                const uint32_t idesc = instr_desc_bf16(2 * kBlockM, n_mma, a_mn, b_mn);
                 const uint32_t a_lbo = a_mn ? kSubBytes : 16u, a_step = a_mn ? 2048u : 32u;
                 const uint32_t b_lbo = b_mn ? kSubBytes : 16u, b_step = b_mn ? 2048u : 32u;
                 const uint32_t acc = tile_no & 1u, aph = (tile_no >> 1) & 1u;
-                if (!mbar_wait_cl(smem_u32(&sh.acc_empty[acc]), aph ^ 1u, abort_flag, status)) break;
+                if (!mbar_wait_cl(smem_u32(&sh.acc_empty[acc]), aph ^ 1u, W)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kAccCols;
-                const uint32_t nkb = (d.k1 - d.k0 + kBlockK - 1) / kBlockK;
+                const uint32_t nkb = (k1 - k0 + kBlockK - 1) / kBlockK;
                 for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                     const uint32_t s = it % kPairStages, ph = (it / kPairStages) & 1u;
-                    if (!mbar_wait_cl(smem_u32(&sh.full[s]), ph, abort_flag, status)) { ok = false; break; }
+                    if (!mbar_wait_cl(smem_u32(&sh.full[s]), ph, W)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = stage_base + s * kPairStageBytes, sb = sa + kPairABytes;
 #pragma unroll
@@ -303,40 +411,46 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
             umma_commit_local_pair(smem_u32(&sh.drain));
             const uint64_t t0 = global_timer_ns();
             while (!mbar_try_wait_cl(smem_u32(&sh.drain), 0u))
-                if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(status, STATUS_TIMEOUT); break; }
+                if (global_timer_ns() - t0 > 2000000000ull) { atomicOr(P.status, STATUS_TIMEOUT); break; }
         }
     } else if (warp >= kEpiWarp0) {
-        // ---- epilogue (both CTAs): own 128 rows of the accumulator -> packed partial block ---------------------
+        // ---- epilogue (both CTAs): the 128 accumulator rows of this CTA's half -> block / C, bookkeeping --------
         const uint32_t group = (warp - kEpiWarp0) / kEpiWarpsPerGroup;
         const uint32_t quad = warp & 3u;
         float* stage_tile = reinterpret_cast<float*>(dyn_smem + (stage_base - smem_u32(dyn_smem)) + kPairStages * kPairStageBytes) +
                             (warp - kEpiWarp0) * kEpiStageFloats;
         const uint32_t sched_empty_leader0 = mapa_shared(smem_u32(&sh.sched_empty[0]), 0u);
         const uint32_t acc_empty_leader = mapa_shared(smem_u32(&sh.acc_empty[group]), 0u);
+        const bool out_bf16 = P.mode & MODE_BF16;
         uint32_t used = 0, tile_no = 0;
         for (uint32_t i = 0;; ++i) {
             const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-            bool ok = mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, abort_flag, status);
+            bool ok = mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, W);
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
-            const uint32_t flags = sh.slot[q].flags, task = sh.slot[q].task, n_mma = sh.slot[q].n_mma;
-            const uint32_t tile_rows = sh.slot[q].rows, cols = sh.slot[q].cols, gemm = sh.slot[q].gemm;
-            // a block of a one-slice GEMM is final: it may go straight to its place in C
-            const bool direct = flags & TILE_DIRECT;
-            const uint32_t ld = direct ? sh.slot[q].ldc : sh.slot[q].ld;
-            const uint64_t out_off = (direct ? sh.slot[q].c_off : sh.slot[q].out_off) + (uint64_t)rank * kBlockM * ld;
+            const TileDesc& sl = sh.slot[q];
+            const uint32_t flags = sl.flags, gemm = sl.gemm, n_mma = sl.n_mma & 0xFFFFu, cols = sl.n_mma >> 16;
+            const uint32_t level = sl.level & 0xFFFFu, nslices = sl.level >> 16, ldc = sl.ldc, n_col = sl.n_col;
+            const TileHalf h = sl.h[rank];
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
             if (flags & TILE_END) break;
             const bool mine = (tile_no & 1u) == group;       // tiles alternate between the two accumulator slots
             ++tile_no;
             if (!mine) continue;
-            const uint32_t rows = rows_of_rank(tile_rows, rank);
-            ok = mbar_wait_cl(smem_u32(&sh.acc_full[group]), used & 1u, abort_flag, status);
+            const uint32_t rows = (flags & (TILE_LIVE0 << rank)) ? h.rows : 0u;
+            // a block of a one-slice GEMM is final: it may go straight to its place in C
+            const bool direct = (P.mode & MODE_DIRECT) && (flags & TILE_SINGLE);
+            const bool to_bf16 = direct && out_bf16;
+            const uint64_t c_off = (uint64_t)h.m_row * ldc + n_col;
+            const uint32_t ld = direct ? ldc : h.ld;
+            const uint64_t out_off = (direct ? c_off : h.out_off) + (uint64_t)(quad * 32u) * ld;
+            ok = mbar_wait_cl(smem_u32(&sh.acc_full[group]), used & 1u, W);
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
             ++used;
             tc_fence_after();
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
-            float* out_blk = (direct ? c_ptrs[gemm] : partials) + out_off + (uint64_t)(quad * 32u) * ld;
+            float* out_f32 = (direct ? static_cast<float*>(P.c_ptrs[gemm]) : P.partials) + out_off;
+            __nv_bfloat16* out_b16 = static_cast<__nv_bfloat16*>(P.c_ptrs[gemm]) + out_off;
             const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
             const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
@@ -356,25 +470,55 @@ exec_pair_kernel(const TileDesc* __restrict__ tiles, uint32_t tile_end, unsigned
                 const uint32_t c0 = c * 32u;
                 if (vec_ok && c0 + 32u <= cols) {
                     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
-                    float* dst = out_blk + c0 + cc;
 #pragma unroll
                     for (uint32_t r = rr; r < 32u; r += 4u) {
                         if (r < rows_here) {
                             const float* src = stage_tile + r * 33 + cc;
-                            *reinterpret_cast<float4*>(dst + (uint64_t)r * ld) = make_float4(src[0], src[1], src[2], src[3]);
+                            if (to_bf16) *reinterpret_cast<uint2*>(out_b16 + (uint64_t)r * ld + c0 + cc) =
+                                             make_uint2(pack_bf16(src[0], src[1]), pack_bf16(src[2], src[3]));
+                            else         *reinterpret_cast<float4*>(out_f32 + (uint64_t)r * ld + c0 + cc) =
+                                             make_float4(src[0], src[1], src[2], src[3]);
                         }
                     }
                 } else if (c0 + lane < cols) {
-                    float* dst = out_blk + c0 + lane;
 #pragma unroll 8
-                    for (uint32_t r = 0; r < rows_here; ++r) dst[(uint64_t)r * ld] = stage_tile[r * 33 + lane];
+                    for (uint32_t r = 0; r < rows_here; ++r) {
+                        const float x = stage_tile[r * 33 + lane];
+                        if (to_bf16) out_b16[(uint64_t)r * ld + c0 + lane] = __float2bfloat16_rn(x);
+                        else         out_f32[(uint64_t)r * ld + c0 + lane] = x;
+                    }
                 }
                 __syncwarp();
             }
             if (rows) {
-                __threadfence();
+                __threadfence();                             // this strip's stores before its arrival is counted
                 __syncwarp();
-                if (lane == 0) atomicAdd(&done[task], 1u);   // one count per warp and 128-row half-tile
+                if (lane == 0) atomicAdd(&P.done[h.task], 1u);   // one count per warp and half-tile
+                if ((P.mode & MODE_FINISH) && !direct && h.fin != kNoFin) {
+                    // the strip of the K-slice that arrives last at the cell sums the cell
+                    unsigned int before = 0;
+                    if (lane == 0) before = atomicAdd(&P.fin_count[h.fin * 4u + quad], 1u);
+                    before = __shfl_sync(0xFFFFFFFFu, before, 0);
+                    if (before + 1u == nslices && rows_here) {
+                        __threadfence();                     // the other slices' stores are visible after their counts
+                        const FinRef* refs = P.fin_refs + __ldg(P.fin_ref0 + h.fin);
+                        void* cb = P.c_ptrs[gemm];
+                        const uint32_t r0 = quad * 32u;
+                        if (nslices <= 2) {
+                            if (out_bf16) finish_strip<2, true>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                            else          finish_strip<2, false>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                        } else if (nslices <= 4) {
+                            if (out_bf16) finish_strip<4, true>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                            else          finish_strip<4, false>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                        } else {
+                            if (out_bf16) finish_strip<8, true>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                            else          finish_strip<8, false>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                        }
+                        __threadfence();
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) atomicSub(&P.level_left[level], 1u);   // after everything this strip had to write
             }
         }
     }
@@ -392,10 +536,8 @@ cudaError_t exec_pair_kernel_prepare() {
     return cudaFuncSetAttribute(exec_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairDynSmem);
 }
 
-cudaError_t launch_exec_pair(uint32_t clusters, const TileDesc* tiles, uint32_t tile_end, unsigned int* ticket,
-                             const CUtensorMap* maps, float* partials, float* const* c_ptrs, uint32_t* done,
-                             unsigned int* status, cudaStream_t st) {
-    exec_pair_kernel<<<2 * clusters, kExecThreads, kPairDynSmem, st>>>(tiles, tile_end, ticket, maps, partials, c_ptrs, done, status);
+cudaError_t launch_exec_pair(uint32_t clusters, const ExecParams& e, cudaStream_t st) {
+    exec_pair_kernel<<<2 * clusters, kExecThreads, kPairDynSmem, st>>>(e);
     return cudaGetLastError();
 }
 

@@ -259,7 +259,7 @@ int validate_common(const cleave_plan_s& p) {
     if (p.gemms.empty()) return CLEAVE_E_INVAL;
     for (const auto& g : p.gemms) {
         if (!g.M || !g.N || !g.K || g.M >= (1u << 31) || g.N >= (1u << 31) || g.K >= (1u << 31)) return CLEAVE_E_INVAL;
-        if (g.transA > 1 || g.transB > 1) return CLEAVE_E_INVAL;
+        if (g.transA > 1 || g.transB > 1 || g.level >= 4096) return CLEAVE_E_INVAL;
     }
     return 0;
 }
@@ -492,13 +492,50 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
 }
 
 // ---- exec work list -----------------------------------------------------------------------------
-// A task is cut into tiles of 256 rows x 256 columns (a pair of CTAs runs one tile: 128 rows and half
-// of the columns each).  Tiles are ordered so that tiles running at the same time share operand
-// panels in L2: by GEMM, K-range, band of 4096 rows, then column, then row.
+// A task is cut into half-tiles of 128 rows x <= 256 columns; two half-tiles with the same GEMM,
+// K-range and columns form a pair, the unit a cluster of two CTAs runs (one CTA per half).  The
+// halves of a pair need not be neighbours nor belong to the same task: in a column strip every
+// block has the same columns, so a block of an odd number of 128-row granules shares a pair with
+// the block below it and no MMA rows stay empty.
+//
+// Order of the pairs (tiles running at the same time share operand panels in L2): by DAG level,
+// GEMM, band of rows, column, row; the K-slices of one cell follow each other when the GEMM's cells
+// can be summed by the exec kernel itself (the block written last then finds the others in L2),
+// otherwise a GEMM is walked K-range by K-range.
+namespace {
+
+struct HalfKey {
+    uint32_t gemm, k0, k1, n_col, cols;
+    bool operator==(const HalfKey& o) const { return gemm == o.gemm && k0 == o.k0 && k1 == o.k1 && n_col == o.n_col && cols == o.cols; }
+};
+struct Half {
+    HalfKey key;
+    TileHalf h;
+    uint32_t kslice;
+};
+
+// widths of the column tiles of a block of beta columns
+void column_tiles(uint32_t beta, std::vector<uint32_t>& w) {
+    w.clear();
+    const uint32_t nt = (uint32_t)cdiv(beta, 256);
+    // full-width tiles first, the remainder last: fewest operand bytes per FLOP
+    for (uint32_t j = 0; j < nt; ++j) w.push_back(std::min(256u, beta - j * 256));
+}
+
+}  // namespace
+
 void build_tiles(cleave_plan_s& p, uint32_t first_task) {
     const uint32_t kBandRows = 4096;
-    const size_t begin = p.tiles.size();
+    const bool original = (first_task == 0);
     p.task_ntiles.resize(p.tasks.size(), 0);
+    if (original) {
+        p.n_levels = 1;
+        for (const auto& g : p.gemms) p.n_levels = std::max<uint32_t>(p.n_levels, (uint32_t)g.level + 1);
+        p.gemm_finishable.assign(p.gemms.size(), 0);
+        p.fin_ref0.clear(); p.fin_refs.clear();
+    }
+    std::vector<Half> halves;
+    std::vector<uint32_t> widths;
     for (uint32_t id = first_task; id < p.tasks.size(); ++id) {
         const cleave_task_t& t = p.tasks[id];
         const cleave_gemm_t& g = p.gemms[t.gemm];
@@ -506,37 +543,105 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
         if ((t.k0 % 64) || ((t.k1 % 64) && t.k1 != g.K) || (g.transA && (t.m0 % 8)) || (!g.transB && (t.n0 % 8)) ||
             (g.lda % 8) || (g.ldb % 8))
             p.exec_unsupported = 1;
-        const uint32_t w = 256;      // full-width tiles first, the remainder last: fewest operand bytes per FLOP
-        const uint32_t nt = (uint32_t)cdiv(beta, w), mt = (uint32_t)cdiv(alpha, 256);
-        p.task_ntiles[id] = nt * (uint32_t)cdiv(alpha, 128);      // bookkeeping counts 128-row half-tiles
-        for (uint32_t ti = 0; ti < mt; ++ti)
-            for (uint32_t tj = 0; tj < nt; ++tj) {
-                TileDesc d;
-                std::memset(&d, 0, sizeof d);
-                d.task = id; d.gemm = t.gemm;
-                d.flags = TILE_VALID | (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN) |
-                          (p.ksplit[t.gemm] == 1 ? TILE_SINGLE : 0u) |
-                          ((!g.transA || g.M % 64 == 0) ? TILE_A_BIG : 0u) | ((g.transB || g.N % 64 == 0) ? TILE_B_BIG : 0u);
-                d.rows = std::min(256u, alpha - ti * 256);
-                d.cols = std::min(w, beta - tj * w);
-                d.n_mma = (d.cols + 15) / 16 * 16;
-                d.m_row = t.m0 + ti * 256;
-                d.n_col = t.n0 + tj * w;
-                d.k0 = t.k0; d.k1 = t.k1;
-                d.ld = beta;
-                d.ldc = g.N;
-                d.c_off = (uint64_t)d.m_row * g.N + d.n_col;
-                d.out_off = t.part_off + (uint64_t)ti * 256 * beta + (uint64_t)tj * w;
-                p.tiles.push_back(d);
+        column_tiles(beta, widths);
+        const uint32_t mh = (uint32_t)cdiv(alpha, 128);
+        p.task_ntiles[id] = mh * (uint32_t)widths.size();      // bookkeeping counts half-tiles
+        for (uint32_t hi = 0; hi < mh; ++hi) {
+            uint32_t col = 0;
+            for (uint32_t wj : widths) {
+                Half x;
+                x.key = HalfKey{t.gemm, t.k0, t.k1, t.n0 + col, wj};
+                x.h.task = id;
+                x.h.m_row = t.m0 + hi * 128;
+                x.h.rows = std::min(128u, alpha - hi * 128);
+                x.h.ld = beta;
+                x.h.out_off = t.part_off + (uint64_t)hi * 128 * beta + col;
+                x.h.fin = kNoFin;
+                x.h.pad = 0;
+                x.kslice = t.kslice;
+                halves.push_back(x);
+                col += wj;
             }
+        }
+    }
+
+    // ---- cells of the in-kernel K-slice sum (original plan only): a GEMM qualifies when every half-tile
+    // position holds exactly one half-tile per K-slice, all of equal shape, and float4 accesses are aligned
+    if (original) {
+        std::vector<std::vector<uint32_t>> by_gemm(p.gemms.size());
+        for (uint32_t i = 0; i < halves.size(); ++i) by_gemm[halves[i].key.gemm].push_back(i);
+        for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
+            const uint32_t S = p.ksplit[gi];
+            if (S < 2 || S > 8 || p.gemms[gi].N % 4) continue;
+            std::vector<uint32_t>& idx = by_gemm[gi];
+            std::sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
+                const Half &x = halves[a], &y = halves[b];
+                if (x.h.m_row != y.h.m_row) return x.h.m_row < y.h.m_row;
+                if (x.key.n_col != y.key.n_col) return x.key.n_col < y.key.n_col;
+                return x.kslice < y.kslice;
+            });
+            bool ok = idx.size() % S == 0;
+            for (size_t c = 0; ok && c < idx.size(); c += S)
+                for (uint32_t s = 0; ok && s < S; ++s) {
+                    const Half &x = halves[idx[c + s]], &x0 = halves[idx[c]];
+                    ok = x.kslice == s && x.h.m_row == x0.h.m_row && x.h.rows == x0.h.rows && x.key.n_col == x0.key.n_col &&
+                         x.key.cols == x0.key.cols && x.key.n_col % 4 == 0 && x.key.cols % 4 == 0 && x.h.ld % 4 == 0 &&
+                         x.h.out_off % 4 == 0;
+                }
+            if (!ok) continue;
+            p.gemm_finishable[gi] = 1;
+            for (size_t c = 0; c < idx.size(); c += S) {
+                const uint32_t cell = (uint32_t)p.fin_ref0.size();
+                p.fin_ref0.push_back((uint32_t)p.fin_refs.size());
+                for (uint32_t s = 0; s < S; ++s) {
+                    Half& x = halves[idx[c + s]];
+                    x.h.fin = cell;
+                    p.fin_refs.push_back(FinRef{x.h.out_off, x.h.ld, x.h.task});
+                }
+            }
+        }
+    }
+
+    // ---- pairs: consecutive half-tiles (by row) of the same GEMM, K-range and columns
+    std::stable_sort(halves.begin(), halves.end(), [](const Half& a, const Half& b) {
+        if (a.key.gemm != b.key.gemm) return a.key.gemm < b.key.gemm;
+        if (a.key.k0 != b.key.k0) return a.key.k0 < b.key.k0;
+        if (a.key.k1 != b.key.k1) return a.key.k1 < b.key.k1;
+        if (a.key.n_col != b.key.n_col) return a.key.n_col < b.key.n_col;
+        if (a.key.cols != b.key.cols) return a.key.cols < b.key.cols;
+        return a.h.m_row < b.h.m_row;
+    });
+    const size_t begin = p.tiles.size();
+    for (size_t i = 0; i < halves.size();) {
+        const Half& x = halves[i];
+        const cleave_gemm_t& g = p.gemms[x.key.gemm];
+        TileDesc d;
+        std::memset(&d, 0, sizeof d);
+        d.gemm = x.key.gemm;
+        d.flags = (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN) | (p.ksplit[d.gemm] == 1 ? TILE_SINGLE : 0u) |
+                  ((!g.transA || g.M % 64 == 0) ? TILE_A_BIG : 0u) | ((g.transB || g.N % 64 == 0) ? TILE_B_BIG : 0u);
+        d.n_col = x.key.n_col;
+        d.n_mma = ((x.key.cols + 15) / 16 * 16) | (x.key.cols << 16);
+        d.k0 = x.key.k0; d.k1 = x.key.k1;
+        d.ldc = g.N;
+        d.level = (uint32_t)g.level | (p.ksplit[d.gemm] << 16);
+        d.h[0] = x.h;
+        // each CTA of the pair loads, multiplies and stores its own half, so any two half-tiles may share a pair
+        if (i + 1 < halves.size() && halves[i + 1].key == x.key) { d.h[1] = halves[i + 1].h; i += 2; }
+        else { d.h[1].task = x.h.task; d.h[1].fin = kNoFin; i += 1; }
+        p.tiles.push_back(d);
     }
     std::stable_sort(p.tiles.begin() + begin, p.tiles.end(), [&](const TileDesc& a, const TileDesc& b) {
+        const uint32_t la = a.level & 0xFFFFu, lb = b.level & 0xFFFFu;
+        if (la != lb) return la < lb;
         if (a.gemm != b.gemm) return a.gemm < b.gemm;
-        if (a.k0 != b.k0) return a.k0 < b.k0;
-        const uint32_t ba = a.m_row / kBandRows, bb = b.m_row / kBandRows;
+        const bool cells = original && p.gemm_finishable[a.gemm];
+        if (!cells && a.k0 != b.k0) return a.k0 < b.k0;
+        const uint32_t ba = a.h[0].m_row / kBandRows, bb = b.h[0].m_row / kBandRows;
         if (ba != bb) return ba < bb;
         if (a.n_col != b.n_col) return a.n_col < b.n_col;
-        return a.m_row < b.m_row;
+        if (a.h[0].m_row != b.h[0].m_row) return a.h[0].m_row < b.h[0].m_row;
+        return a.k0 < b.k0;
     });
 }
 
@@ -627,13 +732,14 @@ int build_assembly(cleave_plan_s& p) {
     std::vector<AsmItem> sorted;
     sorted.reserve(p.asm_items.size());
     for (uint32_t single : {1u, 0u})
-        for (uint32_t cls : {1u, 2u, 4u, 8u, 16u, 32u, 0u}) {
-            const uint32_t item0 = (uint32_t)sorted.size();
-            for (uint32_t gi = 0; gi < p.gemms.size(); ++gi)
-                if (gemm_sp[gi] == cls && (p.ksplit[gi] == 1 ? 1u : 0u) == single)
-                    sorted.insert(sorted.end(), p.asm_items.begin() + first_item[gi], p.asm_items.begin() + first_item[gi + 1]);
-            if (sorted.size() > item0) p.asm_groups.push_back({cls, item0, (uint32_t)sorted.size() - item0, single});
-        }
+        for (uint32_t fin : {1u, 0u})
+            for (uint32_t cls : {1u, 2u, 4u, 8u, 16u, 32u, 0u}) {
+                const uint32_t item0 = (uint32_t)sorted.size();
+                for (uint32_t gi = 0; gi < p.gemms.size(); ++gi)
+                    if (gemm_sp[gi] == cls && (p.ksplit[gi] == 1 ? 1u : 0u) == single && (uint32_t)p.gemm_finishable[gi] == fin)
+                        sorted.insert(sorted.end(), p.asm_items.begin() + first_item[gi], p.asm_items.begin() + first_item[gi + 1]);
+                if (sorted.size() > item0) p.asm_groups.push_back({cls, item0, (uint32_t)sorted.size() - item0, single, fin});
+            }
     p.asm_items.swap(sorted);
     return 0;
 }

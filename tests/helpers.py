@@ -52,24 +52,32 @@ def oracle_operands(w, tensors):
 class GpuRun:
     """Device copies of the operands plus arena and outputs for one workload and plan."""
 
-    def __init__(self, w, tensors, plan, poison=True):
+    def __init__(self, w, tensors, plan, poison=True, bf16_out=False):
         import torch
         self.torch = torch
         self.w, self.plan = w, plan
         dev = torch.device("cuda:0")
         self.dev_tensors = {k: t.to(dev) for k, t in tensors.items()}
+        c_dtype = torch.bfloat16 if bf16_out else torch.float32
+        # tensors the step itself produces (outputs of lower DAG levels that feed higher ones): bf16, NaN until written
+        for k, spec in w.produced.items():
+            self.dev_tensors[k] = torch.full((spec.rows, spec.cols), float("nan"), dtype=torch.bfloat16, device=dev)
         self.A = [self.dev_tensors[g.a_key] for g in w.gemms]
         self.B = [self.dev_tensors[g.b_key] for g in w.gemms]
         self.partials = torch.empty(max(1, plan.arena_elems), dtype=torch.float32, device=dev)
         if poison:
             self.partials.fill_(float("nan"))
-        self.C = [torch.full((g.M, g.N), float("nan"), dtype=torch.float32, device=dev) for g in w.gemms]
+        self.C = [self.dev_tensors[g.out_key] if g.out_key else
+                  torch.full((g.M, g.N), float("nan"), dtype=c_dtype, device=dev) for g in w.gemms]
 
     def exec(self):
         self.plan.exec(self.A, self.B, self.partials)
 
     def exec_fused(self):
         self.plan.exec_fused(self.A, self.B, self.partials, self.C)
+
+    def exec_opts(self, **kw):
+        self.plan.exec_opts(self.A, self.B, self.partials, self.C, **kw)
 
     def assemble(self):
         self.plan.assemble(self.partials, self.C)
@@ -78,8 +86,10 @@ class GpuRun:
         self.plan.reissue(failed, self.A, self.B, self.partials)
 
     def results(self):
+        """fp32 outputs as NumPy arrays; bf16 outputs as their uint16 bit patterns."""
         self.torch.cuda.synchronize()
-        return [c.cpu().numpy() for c in self.C]
+        return [c.cpu().numpy() if c.dtype == self.torch.float32 else
+                c.cpu().view(self.torch.int16).numpy().view(np.uint16) for c in self.C]
 
 
 def assert_within_tolerance(C_gpu, C_ref, bound, rel_fro=1e-3, elem=1e-2, what=""):

@@ -140,14 +140,14 @@ def test_fused_write_out_equals_exec_plus_assemble():
     import paper_2512_22142_b200 as cl
     w = ci.config(4, 8)
     ts = ci.make_tensors(w)
-    p = lib_plan_for(w)
+    p = lib_plan_for(w, kslice_max=512)
     S = [p.ksplit(i) for i in range(p.n_gemms)]
     assert 1 in S and max(S) > 1                      # both kinds of GEMM are present
     base = GpuRun(w, ts, p)
     base.exec(); base.assemble(); p.check_status()
     good = base.results()
 
-    p2 = lib_plan_for(w)
+    p2 = lib_plan_for(w, kslice_max=512)
     run = GpuRun(w, ts, p2)                            # C starts as NaN: nothing may be left unwritten
     launches_two_step = p2.num_launches
     run.exec_fused(); run.assemble(); p2.check_status()

@@ -98,7 +98,7 @@ def test_uniform_and_errors(cl):
     w = ci.config(1)
     p = cl.plan_uniform(w.gemms, 4, 4, 2)
     t = p.tasks()
-    assert p.num_tasks == 32 and p.arena_elems == 393216 and p.num_tiles == 32
+    assert p.num_tasks == 32 and p.arena_elems == 393216 and p.num_tiles == 16   # two 64-row blocks of a column share a pair of CTAs
     assert set(zip(t["m1"] - t["m0"], t["n1"] - t["n0"], t["k1"] - t["k0"])) == {(64, 192, 384)}
     with pytest.raises(cl.CleaveError) as e:
         p.set_drops([32])

@@ -63,9 +63,9 @@ def test_single_slice_is_the_papers_formulation():
 
 
 def test_homogeneous_devices_give_equal_grid():
-    # 16 identical devices, Mg = Ng = 8 (granule 128), S = 1 -> 4 x 4 grid of equal 256 x 256 blocks
+    # 16 identical devices, Mg = Ng = 8, S = 1 -> 4 x 4 grid of equal 256 x 256 blocks
     devs = devices_from_array(ci.homogeneous_devices(16))
-    p = plan([Gemm(1024, 1024, 512)], devs, Opts(gran_m=128, gran_n=128, kslice_max=0))
+    p = plan([Gemm(1024, 1024, 512)], devs, Opts(kslice_max=0))
     assert len(p.tasks) == 16
     assert {(t.alpha, t.beta, t.kappa) for t in p.tasks} == {(256, 256, 512)}
     assert {(t.m0, t.n0) for t in p.tasks} == {(i * 256, j * 256) for i in range(4) for j in range(4)}
@@ -119,14 +119,14 @@ def test_memory_repair_and_infeasible():
 
 def test_auto_ksplit():
     devs = small_devices(8, 1, 1 << 28, 1 << 30)
-    assert plan([Gemm(512, 256, 8192)], devs[:4], Opts()).ksplit == [2]        # depth cap 4096
-    assert plan([Gemm(512, 256, 11008)], devs[:4], Opts()).ksplit == [3]
-    assert plan([Gemm(512, 256, 4096)], devs[:4], Opts()).ksplit == [1]
-    assert plan([Gemm(512, 256, 4096)], devs[:4], Opts(kslice_max=2048)).ksplit == [2]
+    assert plan([Gemm(256, 256, 8192)], devs[:4], Opts()).ksplit == [2]        # depth cap 4096
+    assert plan([Gemm(256, 256, 11008)], devs[:4], Opts()).ksplit == [3]
+    assert plan([Gemm(256, 256, 4096)], devs[:4], Opts()).ksplit == [1]
+    assert plan([Gemm(256, 256, 4096)], devs[:4], Opts(kslice_max=2048)).ksplit == [2]
     # more devices than output cells -> split K so that all can work (2x2 cells, 8 devices)
-    assert plan([Gemm(512, 256, 512)], devs, Opts()).ksplit == [2]
+    assert plan([Gemm(256, 256, 512)], devs, Opts()).ksplit == [2]
     # K-slices are consecutive, granule aligned, sizes differ by at most one granule
-    p = plan([Gemm(512, 256, 11008)], devs[:4], Opts())
+    p = plan([Gemm(256, 256, 11008)], devs[:4], Opts())
     ranges = sorted({(t.k0, t.k1) for t in p.tasks})
     assert ranges == [(0, 3712), (3712, 7424), (7424, 11008)]
 
