@@ -262,6 +262,8 @@ def run_ours(args):
     opts = {}
     if args.kslice_max is not None:
         opts["kslice_max"] = args.kslice_max
+    if args.gran_m is not None:
+        opts["gran_m"] = args.gran_m
     t0 = time.perf_counter()
     tensors = ci.make_tensors(w, pin=True)
     gen_s = time.perf_counter() - t0
@@ -278,7 +280,8 @@ def run_ours(args):
     flops = float(w.flops)
     S = [plan.ksplit(i) for i in range(len(w.gemms))]
     # bytes the assembly kernels move: GEMMs with one K-slice are finished by the exec kernel in fused mode
-    asm_bytes = float(sum((S[i] + 1) * g.M * g.N * 4 for i, g in enumerate(w.gemms) if args.two_step or S[i] > 1))
+    in_kernel = [(not args.two_step) and (S[i] == 1 or (not args.no_finish and plan.finishable(i))) for i in range(len(w.gemms))]
+    asm_bytes = float(sum((S[i] + 1) * g.M * g.N * 4 for i, g in enumerate(w.gemms) if not in_kernel[i]))
 
     def barrier():
         if dist is not None:
@@ -294,7 +297,7 @@ def run_ours(args):
         if args.two_step:
             plan.exec(A, B, partials)
         else:
-            plan.exec_fused(A, B, partials, C)
+            plan.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish)
 
     for _ in range(args.warmup):
         run_exec()
@@ -509,6 +512,8 @@ def main():
     ap.add_argument("--no-churn", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--two-step", action="store_true", help="cleave_exec + full cleave_assemble instead of the fused write-out")
+    ap.add_argument("--no-finish", action="store_true", help="fused write-out of one-slice GEMMs only; K-split GEMMs go through cleave_assemble")
+    ap.add_argument("--gran-m", type=int, default=None, help="row granule of the planner (default 128)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -24,11 +24,14 @@
 //
 // Write-out (epilogue warps, each owning a strip of 32 accumulator rows).  The strip always goes to
 // the task's packed block in the arena, or, for a GEMM with one K-slice under MODE_DIRECT, to its
-// place in C.  Under MODE_FINISH a strip of a GEMM with several K-slices then counts its arrival at
-// its cell; the strip that arrives last reads the cell's blocks of all K-slices back (they are in
-// L2: the slices of a cell follow each other in the work list), sums them in the fixed balanced-tree
-// order -- the order does not depend on which block arrived last -- and writes C.  Under MODE_BF16
-// values written to C are rounded to bf16.
+// place in C.  Under MODE_FINISH a strip of a GEMM with several K-slices counts its arrival at its
+// cell after its block is stored, and the strip that is last sums the cell's blocks of all K-slices in
+// the fixed balanced-tree order -- the order does not depend on which block was last -- and writes C.
+// Usually a strip already finds every other slice's block stored when its tile is handed out (a GEMM is
+// walked K-range by K-range): it then asks for those blocks to be brought into L2 while its own MMAs
+// still run, and adds them to its accumulator values on their way out (no second pass over its own
+// block).  A strip that only turns out to be last after storing its block reads all blocks back.
+// Under MODE_BF16 values written to C are rounded to bf16.
 //
 // DAG levels: tiles are ordered by level, and before the scheduler hands out the first tile of a
 // level it waits until every strip of the lower levels has been written (a counter per level that
@@ -189,12 +192,12 @@ struct __align__(16) PairShared {
 
 // Sum of the SP (slice count padded to a power of two) blocks of a cell for one 32-row strip, in
 // the order of the assembly kernel: balanced pairwise tree over adjacent slices, missing slices
-// contribute +0.0f.  One float4 per lane and step, four steps in flight.
+// contribute +0.0f.  One float4 per lane and step, four to eight steps in flight.
 template <int SP, bool BF16>
 __device__ __forceinline__ void finish_strip(const FinRef* __restrict__ refs, uint32_t nslices, const float* __restrict__ partials,
                                              uint32_t row0, uint32_t nrows, uint32_t cols, void* c_base, uint64_t c_off,
                                              uint32_t ldc, uint32_t lane) {
-    constexpr int U = 4;
+    constexpr int U = SP <= 2 ? 8 : (SP <= 4 ? 4 : 2);
     const float* src[SP];
     uint32_t ld[SP];
 #pragma unroll
@@ -233,6 +236,59 @@ __device__ __forceinline__ void finish_strip(const FinRef* __restrict__ refs, ui
             if (BF16) *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(c_base) + at) =
                           make_uint2(pack_bf16(acc[u].x, acc[u].y), pack_bf16(acc[u].z, acc[u].w));
             else      *reinterpret_cast<float4*>(static_cast<float*>(c_base) + at) = acc[u];
+        }
+    }
+}
+
+// One 32 x 32 chunk of a strip whose cell is complete but for this block: the staged accumulator
+// values (own K-slice `mine`) go to the block in the arena as always, and, added to the other slices'
+// values in the fixed tree order, to C.  Lanes: 8 per row segment of 32 columns, 4 rows per step.
+template <int SP, bool BF16>
+__device__ __forceinline__ void store_chunk_summed(const float* stage_tile, const FinRef* __restrict__ refs, uint32_t nslices,
+                                                   uint32_t mine, const float* __restrict__ partials, float* own_blk,
+                                                   uint32_t own_ld, uint32_t row0, uint32_t rows_here, uint32_t c0, uint32_t cols,
+                                                   void* c_base, uint64_t c_off, uint32_t ldc, uint32_t lane) {
+    constexpr int RB = SP <= 2 ? 4 : (SP <= 4 ? 2 : 1);      // rows per lane whose loads are in flight together
+    const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
+    if (c0 + cc >= cols) rows_here = 0;                      // ragged last chunk (columns come in fours)
+    const float* src[SP];
+    uint32_t ld[SP];
+#pragma unroll
+    for (int s = 0; s < SP; ++s) {
+        if ((uint32_t)s < nslices && (uint32_t)s != mine) { const FinRef rf = refs[s]; src[s] = partials + rf.off + (uint64_t)row0 * rf.ld + c0 + cc; ld[s] = rf.ld; }
+        else { src[s] = nullptr; ld[s] = 0; }
+    }
+#pragma unroll
+    for (int b = 0; b < 8; b += RB) {
+        float4 v[RB][SP];
+#pragma unroll
+        for (int x = 0; x < RB; ++x) {
+            const uint32_t r = rr + 4u * (uint32_t)(b + x);
+#pragma unroll
+            for (int s = 0; s < SP; ++s) {
+                v[x][s] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < rows_here && src[s]) v[x][s] = ld_cg_f4(src[s] + (uint64_t)r * ld[s]);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < RB; ++x) {
+            const uint32_t r = rr + 4u * (uint32_t)(b + x);
+            if (r >= rows_here) continue;
+            const float* st = stage_tile + r * 33 + cc;
+            const float4 own = make_float4(st[0], st[1], st[2], st[3]);
+            *reinterpret_cast<float4*>(own_blk + (uint64_t)r * own_ld + c0 + cc) = own;
+#pragma unroll
+            for (int s = 0; s < SP; ++s) if ((uint32_t)s == mine) v[x][s] = own;
+#pragma unroll
+            for (int w = 1; w < SP; w *= 2)
+#pragma unroll
+                for (int s = 0; s < SP; s += 2 * w) {
+                    v[x][s].x += v[x][s + w].x; v[x][s].y += v[x][s + w].y; v[x][s].z += v[x][s + w].z; v[x][s].w += v[x][s + w].w;
+                }
+            const uint64_t at = c_off + (uint64_t)(row0 + r) * ldc + c0 + cc;
+            if (BF16) *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(c_base) + at) =
+                          make_uint2(pack_bf16(v[x][0].x, v[x][0].y), pack_bf16(v[x][0].z, v[x][0].w));
+            else      *reinterpret_cast<float4*>(static_cast<float*>(c_base) + at) = v[x][0];
         }
     }
 }
@@ -429,7 +485,8 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
             const TileDesc& sl = sh.slot[q];
             const uint32_t flags = sl.flags, gemm = sl.gemm, n_mma = sl.n_mma & 0xFFFFu, cols = sl.n_mma >> 16;
-            const uint32_t level = sl.level & 0xFFFFu, nslices = sl.level >> 16, ldc = sl.ldc, n_col = sl.n_col;
+            const uint32_t level = sl.level & 0xFFFFu, nslices = (sl.level >> 16) & 0xFFu, kslice = sl.level >> 24;
+            const uint32_t ldc = sl.ldc, n_col = sl.n_col;
             const TileHalf h = sl.h[rank];
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
@@ -438,12 +495,37 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             ++tile_no;
             if (!mine) continue;
             const uint32_t rows = (flags & (TILE_LIVE0 << rank)) ? h.rows : 0u;
+            const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
+            const uint32_t row0 = quad * 32u;
             // a block of a one-slice GEMM is final: it may go straight to its place in C
             const bool direct = (P.mode & MODE_DIRECT) && (flags & TILE_SINGLE);
             const bool to_bf16 = direct && out_bf16;
+            const bool cell = (P.mode & MODE_FINISH) && !direct && h.fin != kNoFin && rows;
             const uint64_t c_off = (uint64_t)h.m_row * ldc + n_col;
             const uint32_t ld = direct ? ldc : h.ld;
-            const uint64_t out_off = (direct ? c_off : h.out_off) + (uint64_t)(quad * 32u) * ld;
+            const uint64_t out_off = (direct ? c_off : h.out_off) + (uint64_t)row0 * ld;
+            // Is every other K-slice's block of this strip's cell stored already?  Then this strip is the last
+            // one: start bringing those blocks into L2 now, while the MMAs of this tile still run.
+            bool sum_now = false;
+            const FinRef* refs = nullptr;
+            if (cell) {
+                unsigned int arrived;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(P.fin_count + h.fin * 4u + quad) : "memory");
+                sum_now = __shfl_sync(0xFFFFFFFFu, arrived, 0) + 1u == nslices;
+                refs = P.fin_refs + __ldg(P.fin_ref0 + h.fin);
+                if (sum_now && rows_here) {
+                    const uint32_t lines_per_row = (cols * 4u + 127u) / 128u;
+                    for (uint32_t s = 0; s < nslices; ++s) {
+                        if (s == kslice) continue;
+                        const FinRef rf = refs[s];
+                        const float* base = P.partials + rf.off + (uint64_t)row0 * rf.ld;
+                        for (uint32_t x = lane; x < rows_here * lines_per_row; x += 32u) {
+                            const uint32_t r = x / lines_per_row, seg = x - r * lines_per_row;
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (uint64_t)r * rf.ld + seg * 32u));
+                        }
+                    }
+                }
+            }
             ok = mbar_wait_cl(smem_u32(&sh.acc_full[group]), used & 1u, W);
             if (!__all_sync(0xFFFFFFFFu, ok)) break;
             ++used;
@@ -451,7 +533,6 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
             float* out_f32 = (direct ? static_cast<float*>(P.c_ptrs[gemm]) : P.partials) + out_off;
             __nv_bfloat16* out_b16 = static_cast<__nv_bfloat16*>(P.c_ptrs[gemm]) + out_off;
-            const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
             const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
             for (uint32_t c = 0; c < nchunk; ++c) {
@@ -468,7 +549,20 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
                 __syncwarp();
                 const uint32_t c0 = c * 32u;
-                if (vec_ok && c0 + 32u <= cols) {
+                if (sum_now) {
+                    // (cells exist only where float4 accesses are aligned and columns come in fours)
+                    void* cb = P.c_ptrs[gemm];
+                    if (nslices <= 2) {
+                        if (out_bf16) store_chunk_summed<2, true>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                        else          store_chunk_summed<2, false>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                    } else if (nslices <= 4) {
+                        if (out_bf16) store_chunk_summed<4, true>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                        else          store_chunk_summed<4, false>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                    } else {
+                        if (out_bf16) store_chunk_summed<8, true>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                        else          store_chunk_summed<8, false>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                    }
+                } else if (vec_ok && c0 + 32u <= cols) {
                     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
 #pragma unroll
                     for (uint32_t r = rr; r < 32u; r += 4u) {
@@ -494,28 +588,26 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 __threadfence();                             // this strip's stores before its arrival is counted
                 __syncwarp();
                 if (lane == 0) atomicAdd(&P.done[h.task], 1u);   // one count per warp and half-tile
-                if ((P.mode & MODE_FINISH) && !direct && h.fin != kNoFin) {
-                    // the strip of the K-slice that arrives last at the cell sums the cell
+                if (cell) {
                     unsigned int before = 0;
                     if (lane == 0) before = atomicAdd(&P.fin_count[h.fin * 4u + quad], 1u);
                     before = __shfl_sync(0xFFFFFFFFu, before, 0);
-                    if (before + 1u == nslices && rows_here) {
+                    // not known to be last when it started, but last all the same: read every block back and sum
+                    if (!sum_now && before + 1u == nslices && rows_here) {
                         __threadfence();                     // the other slices' stores are visible after their counts
-                        const FinRef* refs = P.fin_refs + __ldg(P.fin_ref0 + h.fin);
                         void* cb = P.c_ptrs[gemm];
-                        const uint32_t r0 = quad * 32u;
                         if (nslices <= 2) {
-                            if (out_bf16) finish_strip<2, true>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
-                            else          finish_strip<2, false>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                            if (out_bf16) finish_strip<2, true>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
+                            else          finish_strip<2, false>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
                         } else if (nslices <= 4) {
-                            if (out_bf16) finish_strip<4, true>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
-                            else          finish_strip<4, false>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                            if (out_bf16) finish_strip<4, true>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
+                            else          finish_strip<4, false>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
                         } else {
-                            if (out_bf16) finish_strip<8, true>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
-                            else          finish_strip<8, false>(refs, nslices, P.partials, r0, rows_here, cols, cb, c_off, ldc, lane);
+                            if (out_bf16) finish_strip<8, true>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
+                            else          finish_strip<8, false>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
                         }
-                        __threadfence();
                     }
+                    if (sum_now || before + 1u == nslices) __threadfence();    // the sums, before the level counts this strip
                 }
                 __syncwarp();
                 if (lane == 0) atomicSub(&P.level_left[level], 1u);   // after everything this strip had to write

@@ -31,7 +31,7 @@ struct TileDesc {
     uint32_t n_mma;     // bits 0-15: MMA N extent (columns rounded up to 16); bits 16-31: valid columns (1..256)
     uint32_t k0, k1;
     uint32_t ldc;       // leading dimension of the GEMM's C (= N)
-    uint32_t level;     // bits 0-15: DAG level of the GEMM; bits 16-31: number of K-slices of the GEMM
+    uint32_t level;     // bits 0-15: DAG level of the GEMM; bits 16-23: its number of K-slices; bits 24-31: this K-slice
     TileHalf h[2];
 };
 static_assert(sizeof(TileDesc) == 96, "TileDesc must be 96 bytes");
