@@ -1,6 +1,6 @@
 // CUDA kernels of the Cleave hot path for sm_100a.
 //
-//   arm_queue_kernel    marks each half of every work-list entry runnable or skipped (dropped /
+//   arm_queue_kernel    marks each quadrant of every work-list entry runnable or skipped (dropped /
 //                       superseded task), clears the bookkeeping of the tasks about to run, counts
 //                       the strips each DAG level has to finish, resets the ticket
 //   (the grouped GEMM itself, exec_pair_kernel, lives in kernels_pair.cu)
@@ -32,22 +32,28 @@ __global__ void arm_queue_kernel(const ArmParams a) {
     TileDesc& d = a.tiles[t];
     uint32_t f = d.flags & ~(uint32_t)(TILE_LIVE0 | TILE_LIVE1);
     const bool direct = (a.mode & MODE_DIRECT) && (f & TILE_SINGLE);
-    const uint32_t cols = d.n_mma >> 16;
-    uint32_t live = 0;
+    const uint32_t cols = d.n_mma >> 16, split = d.split;
     const uint32_t level = d.level & 0xFFFFu;
     const bool in_range = level >= a.level_begin && level < a.level_end;
+    uint32_t live = 0;
     for (uint32_t r = 0; r < 2; ++r) {
-        const TileHalf& h = d.h[r];
-        if (h.rows == 0 || !in_range) continue;
-        a.done[h.task] = 0;                              // every tile of the task writes the same value
-        if (a.dropped[h.task] || (a.tasks[h.task].flags & CLEAVE_TASK_SUPERSEDED)) continue;
-        // range check of the block the half-tile will write: one that would leave the arena is not run
-        if (!direct && h.out_off + (unsigned long long)(h.rows - 1) * h.ld + cols > a.arena_elems) {
-            atomicOr(a.status, STATUS_BOUNDS);
-            continue;
+        TileHalf& h = d.h[r];
+        for (uint32_t q = 0; q < 2; ++q) {
+            TileSeg& sg = h.seg[q];
+            sg.live = 0;
+            const uint32_t width = q == 0 ? min(split, cols) : (cols > split ? cols - split : 0u);
+            if (h.rows == 0 || width == 0 || !in_range) continue;
+            a.done[sg.task] = 0;                         // every quadrant of the task writes the same value
+            if (a.dropped[sg.task] || (a.tasks[sg.task].flags & CLEAVE_TASK_SUPERSEDED)) continue;
+            // range check of what the quadrant will write: one that would leave the arena is not run
+            if (!direct && sg.out_off + (unsigned long long)(h.rows - 1) * sg.ld + width > a.arena_elems) {
+                atomicOr(a.status, STATUS_BOUNDS);
+                continue;
+            }
+            sg.live = 1;
+            f |= TILE_LIVE0 << r;
+            ++live;
         }
-        f |= TILE_LIVE0 << r;
-        ++live;
     }
     d.flags = f;
     if (live) atomicAdd(&a.level_left[level], live * (uint32_t)kEpiWarpsPerGroup);

@@ -248,6 +248,8 @@ __device__ __forceinline__ void store_chunk_summed(const float* stage_tile, cons
                                                    uint32_t mine, const float* __restrict__ partials, float* own_blk,
                                                    uint32_t own_ld, uint32_t row0, uint32_t rows_here, uint32_t c0, uint32_t cols,
                                                    void* c_base, uint64_t c_off, uint32_t ldc, uint32_t lane) {
+    // own_blk: the quadrant's (row0, 0) in this task's block; c0: first column of the chunk inside the quadrant;
+    // cols: the quadrant's columns; c_off: offset of the quadrant's (0, 0) in C
     constexpr int RB = SP <= 2 ? 4 : (SP <= 4 ? 2 : 1);      // rows per lane whose loads are in flight together
     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
     if (c0 + cc >= cols) rows_here = 0;                      // ragged last chunk (columns come in fours)
@@ -486,7 +488,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             const TileDesc& sl = sh.slot[q];
             const uint32_t flags = sl.flags, gemm = sl.gemm, n_mma = sl.n_mma & 0xFFFFu, cols = sl.n_mma >> 16;
             const uint32_t level = sl.level & 0xFFFFu, nslices = (sl.level >> 16) & 0xFFu, kslice = sl.level >> 24;
-            const uint32_t ldc = sl.ldc, n_col = sl.n_col;
+            const uint32_t ldc = sl.ldc, n_col = sl.n_col, split = sl.split;
             const TileHalf h = sl.h[rank];
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
@@ -500,28 +502,32 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             // a block of a one-slice GEMM is final: it may go straight to its place in C
             const bool direct = (P.mode & MODE_DIRECT) && (flags & TILE_SINGLE);
             const bool to_bf16 = direct && out_bf16;
-            const bool cell = (P.mode & MODE_FINISH) && !direct && h.fin != kNoFin && rows;
-            const uint64_t c_off = (uint64_t)h.m_row * ldc + n_col;
-            const uint32_t ld = direct ? ldc : h.ld;
-            const uint64_t out_off = (direct ? c_off : h.out_off) + (uint64_t)row0 * ld;
-            // Is every other K-slice's block of this strip's cell stored already?  Then this strip is the last
-            // one: start bringing those blocks into L2 now, while the MMAs of this tile still run.
-            bool sum_now = false;
-            const FinRef* refs = nullptr;
-            if (cell) {
-                unsigned int arrived;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(P.fin_count + h.fin * 4u + quad) : "memory");
-                sum_now = __shfl_sync(0xFFFFFFFFu, arrived, 0) + 1u == nslices;
-                refs = P.fin_refs + __ldg(P.fin_ref0 + h.fin);
-                if (sum_now && rows_here) {
-                    const uint32_t lines_per_row = (cols * 4u + 127u) / 128u;
-                    for (uint32_t s = 0; s < nslices; ++s) {
-                        if (s == kslice) continue;
-                        const FinRef rf = refs[s];
-                        const float* base = P.partials + rf.off + (uint64_t)row0 * rf.ld;
-                        for (uint32_t x = lane; x < rows_here * lines_per_row; x += 32u) {
-                            const uint32_t r = x / lines_per_row, seg = x - r * lines_per_row;
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (uint64_t)r * rf.ld + seg * 32u));
+            const uint64_t c_off = (uint64_t)h.m_row * ldc + n_col;            // the half-tile's (0, 0) in C
+            // the one or two column segments of the half-tile: quadrants of possibly different tasks
+            const uint32_t width[2] = {min(split, cols), cols > split ? cols - split : 0u};
+            bool cell[2], sum_now[2] = {false, false};
+            const FinRef* refs[2] = {nullptr, nullptr};
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const TileSeg& sg = h.seg[q];
+                cell[q] = rows && sg.live && width[q] && (P.mode & MODE_FINISH) && !direct && sg.fin != kNoFin;
+                // Is every other K-slice's block of this strip's cell stored already?  Then this strip is the last
+                // one: start bringing those blocks into L2 now, while the MMAs of this tile still run.
+                if (cell[q]) {
+                    unsigned int arrived;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(P.fin_count + sg.fin * 4u + quad) : "memory");
+                    sum_now[q] = __shfl_sync(0xFFFFFFFFu, arrived, 0) + 1u == nslices;
+                    refs[q] = P.fin_refs + __ldg(P.fin_ref0 + sg.fin);
+                    if (sum_now[q] && rows_here) {
+                        const uint32_t lines_per_row = (width[q] * 4u + 127u) / 128u;
+                        for (uint32_t s = 0; s < nslices; ++s) {
+                            if (s == kslice) continue;
+                            const FinRef rf = refs[q][s];
+                            const float* base = P.partials + rf.off + (uint64_t)row0 * rf.ld;
+                            for (uint32_t x = lane; x < rows_here * lines_per_row; x += 32u) {
+                                const uint32_t r = x / lines_per_row, seg = x - r * lines_per_row;
+                                asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (uint64_t)r * rf.ld + seg * 32u));
+                            }
                         }
                     }
                 }
@@ -531,9 +537,6 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             ++used;
             tc_fence_after();
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
-            float* out_f32 = (direct ? static_cast<float*>(P.c_ptrs[gemm]) : P.partials) + out_off;
-            __nv_bfloat16* out_b16 = static_cast<__nv_bfloat16*>(P.c_ptrs[gemm]) + out_off;
-            const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
             for (uint32_t c = 0; c < nchunk; ++c) {
                 uint32_t v[32];
@@ -544,42 +547,52 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
                 }
-                if (rows_here == 0) continue;                // warp-uniform
+                const uint32_t q = (c * 32u >= split) ? 1u : 0u;             // (split is a multiple of 32 when a second segment exists)
+                const TileSeg& sg = h.seg[q];
+                if (rows_here == 0 || !sg.live || c * 32u >= cols) continue; // warp-uniform
 #pragma unroll
                 for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
                 __syncwarp();
-                const uint32_t c0 = c * 32u;
-                if (sum_now) {
+                const uint32_t ct = c * 32u;                 // chunk's first column in the half-tile ...
+                const uint32_t c0 = ct - (q ? split : 0u);   // ... and in its quadrant
+                const uint32_t ld = direct ? ldc : sg.ld;
+                const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg.out_off + (uint64_t)row0 * sg.ld + c0;
+                float* out_f32 = (direct ? static_cast<float*>(P.c_ptrs[gemm]) : P.partials) + out_off;
+                __nv_bfloat16* out_b16 = static_cast<__nv_bfloat16*>(P.c_ptrs[gemm]) + out_off;
+                const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
+                if (sum_now[q]) {
                     // (cells exist only where float4 accesses are aligned and columns come in fours)
                     void* cb = P.c_ptrs[gemm];
+                    const uint64_t cq = c_off + (q ? split : 0u);
+                    float* own = P.partials + sg.out_off + (uint64_t)row0 * sg.ld;
                     if (nslices <= 2) {
-                        if (out_bf16) store_chunk_summed<2, true>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
-                        else          store_chunk_summed<2, false>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                        if (out_bf16) store_chunk_summed<2, true>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
+                        else          store_chunk_summed<2, false>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
                     } else if (nslices <= 4) {
-                        if (out_bf16) store_chunk_summed<4, true>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
-                        else          store_chunk_summed<4, false>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                        if (out_bf16) store_chunk_summed<4, true>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
+                        else          store_chunk_summed<4, false>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
                     } else {
-                        if (out_bf16) store_chunk_summed<8, true>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
-                        else          store_chunk_summed<8, false>(stage_tile, refs, nslices, kslice, P.partials, out_f32, ld, row0, rows_here, c0, cols, cb, c_off, ldc, lane);
+                        if (out_bf16) store_chunk_summed<8, true>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
+                        else          store_chunk_summed<8, false>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
                     }
-                } else if (vec_ok && c0 + 32u <= cols) {
+                } else if (vec_ok && ct + 32u <= cols) {
                     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
 #pragma unroll
                     for (uint32_t r = rr; r < 32u; r += 4u) {
                         if (r < rows_here) {
                             const float* src = stage_tile + r * 33 + cc;
-                            if (to_bf16) *reinterpret_cast<uint2*>(out_b16 + (uint64_t)r * ld + c0 + cc) =
+                            if (to_bf16) *reinterpret_cast<uint2*>(out_b16 + (uint64_t)r * ld + cc) =
                                              make_uint2(pack_bf16(src[0], src[1]), pack_bf16(src[2], src[3]));
-                            else         *reinterpret_cast<float4*>(out_f32 + (uint64_t)r * ld + c0 + cc) =
+                            else         *reinterpret_cast<float4*>(out_f32 + (uint64_t)r * ld + cc) =
                                              make_float4(src[0], src[1], src[2], src[3]);
                         }
                     }
-                } else if (c0 + lane < cols) {
+                } else if (ct + lane < cols) {
 #pragma unroll 8
                     for (uint32_t r = 0; r < rows_here; ++r) {
                         const float x = stage_tile[r * 33 + lane];
-                        if (to_bf16) out_b16[(uint64_t)r * ld + c0 + lane] = __float2bfloat16_rn(x);
-                        else         out_f32[(uint64_t)r * ld + c0 + lane] = x;
+                        if (to_bf16) out_b16[(uint64_t)r * ld + lane] = __float2bfloat16_rn(x);
+                        else         out_f32[(uint64_t)r * ld + lane] = x;
                     }
                 }
                 __syncwarp();
@@ -587,30 +600,37 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             if (rows) {
                 __threadfence();                             // this strip's stores before its arrival is counted
                 __syncwarp();
-                if (lane == 0) atomicAdd(&P.done[h.task], 1u);   // one count per warp and half-tile
-                if (cell) {
+                uint32_t n_live = 0;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const TileSeg& sg = h.seg[q];
+                    if (!sg.live || !width[q]) continue;
+                    ++n_live;
+                    if (lane == 0) atomicAdd(&P.done[sg.task], 1u);   // one count per warp and quadrant
+                    if (!cell[q]) continue;
                     unsigned int before = 0;
-                    if (lane == 0) before = atomicAdd(&P.fin_count[h.fin * 4u + quad], 1u);
+                    if (lane == 0) before = atomicAdd(&P.fin_count[sg.fin * 4u + quad], 1u);
                     before = __shfl_sync(0xFFFFFFFFu, before, 0);
                     // not known to be last when it started, but last all the same: read every block back and sum
-                    if (!sum_now && before + 1u == nslices && rows_here) {
+                    if (!sum_now[q] && before + 1u == nslices && rows_here) {
                         __threadfence();                     // the other slices' stores are visible after their counts
                         void* cb = P.c_ptrs[gemm];
+                        const uint64_t cq = c_off + (q ? split : 0u);
                         if (nslices <= 2) {
-                            if (out_bf16) finish_strip<2, true>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
-                            else          finish_strip<2, false>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
+                            if (out_bf16) finish_strip<2, true>(refs[q], nslices, P.partials, row0, rows_here, width[q], cb, cq, ldc, lane);
+                            else          finish_strip<2, false>(refs[q], nslices, P.partials, row0, rows_here, width[q], cb, cq, ldc, lane);
                         } else if (nslices <= 4) {
-                            if (out_bf16) finish_strip<4, true>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
-                            else          finish_strip<4, false>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
+                            if (out_bf16) finish_strip<4, true>(refs[q], nslices, P.partials, row0, rows_here, width[q], cb, cq, ldc, lane);
+                            else          finish_strip<4, false>(refs[q], nslices, P.partials, row0, rows_here, width[q], cb, cq, ldc, lane);
                         } else {
-                            if (out_bf16) finish_strip<8, true>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
-                            else          finish_strip<8, false>(refs, nslices, P.partials, row0, rows_here, cols, cb, c_off, ldc, lane);
+                            if (out_bf16) finish_strip<8, true>(refs[q], nslices, P.partials, row0, rows_here, width[q], cb, cq, ldc, lane);
+                            else          finish_strip<8, false>(refs[q], nslices, P.partials, row0, rows_here, width[q], cb, cq, ldc, lane);
                         }
                     }
-                    if (sum_now || before + 1u == nslices) __threadfence();    // the sums, before the level counts this strip
+                    if (sum_now[q] || before + 1u == nslices) __threadfence();    // the sums, before the level counts this strip
                 }
                 __syncwarp();
-                if (lane == 0) atomicSub(&P.level_left[level], 1u);   // after everything this strip had to write
+                if (lane == 0 && n_live) atomicSub(&P.level_left[level], n_live);   // after everything this strip had to write
             }
         }
     }

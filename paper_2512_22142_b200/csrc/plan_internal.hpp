@@ -10,19 +10,26 @@
 namespace cleave {
 
 // Work unit of the exec kernel: one pair of half-tiles.  A half-tile is <= 128 rows x <= 256 columns
-// of one task's output block over the task's whole K-range; the two halves of a pair are run by the
-// two CTAs of a cluster with one M = 256 MMA stream, so they share the GEMM, the K-range and the
-// columns, but each has its own rows (they may belong to different tasks: any two blocks of a
-// column strip can fill a pair, so blocks made of an odd number of 128-row granules waste nothing).
-// 96 bytes, read by the kernel's scheduler warp with six 16-byte loads.
-struct TileHalf {
+// of a GEMM's output over one K-range; the two halves of a pair are run by the two CTAs of a cluster
+// with one M = 256 MMA stream, so they share the GEMM, the K-range and the columns, but each has its
+// own rows.  The columns of a half-tile fall into one or two segments (the second starts at column
+// `split`), and every (half, segment) quadrant belongs to one task: it is stored into that task's
+// packed block and counted in that task's bookkeeping.  Where all block edges of a GEMM lie on
+// multiples of 128 the GEMM is tiled on a global grid of 256 x 256 pairs whatever the blocks'
+// shapes, each quadrant being the 128 x 128 cell of whichever task owns it there; otherwise every
+// task is cut into half-tiles of its own (one segment each) and half-tiles with equal columns share
+// a pair.  160 bytes, read by the kernel's scheduler warp with ten 16-byte loads.
+struct TileSeg {
     uint32_t task;      // owning task (bookkeeping)
+    uint32_t ld;        // leading dimension of the task's packed block (= beta)
+    uint64_t out_off;   // fp32 element offset of the quadrant's (0,0) in the arena
+    uint32_t fin;       // cell of the in-kernel K-slice sum (kNoFin: none)
+    uint32_t live;      // (set per launch) the quadrant runs: its task is neither dropped nor superseded
+};
+struct TileHalf {
     uint32_t m_row;     // first row of the half-tile in op(A)
     uint32_t rows;      // valid rows (0..128); 0 = the pair has no second half
-    uint32_t ld;        // leading dimension of the task's packed block (= beta)
-    uint64_t out_off;   // fp32 element offset of the half-tile's (0,0) in the arena
-    uint32_t fin;       // cell of the in-kernel K-slice sum (kNoFin: none)
-    uint32_t pad;
+    TileSeg seg[2];     // columns [0, split) and [split, cols); seg[1] unused when split == cols
 };
 struct TileDesc {
     uint32_t gemm;
@@ -33,11 +40,13 @@ struct TileDesc {
     uint32_t ldc;       // leading dimension of the GEMM's C (= N)
     uint32_t level;     // bits 0-15: DAG level of the GEMM; bits 16-23: its number of K-slices; bits 24-31: this K-slice
     TileHalf h[2];
+    uint32_t split;     // first column of the second segment (a multiple of 32), or the number of columns
+    uint32_t pad[3];
 };
-static_assert(sizeof(TileDesc) == 96, "TileDesc must be 96 bytes");
+static_assert(sizeof(TileDesc) == 160, "TileDesc must be 160 bytes");
 constexpr uint32_t kNoFin = 0xFFFFFFFFu;
 
-// LIVE0 / LIVE1: (set per launch) half 0 / 1 runs (its task is neither dropped nor superseded)
+// LIVE0 / LIVE1: (set per launch) half 0 / 1 has a quadrant that runs
 // A_MN / B_MN: the operand is stored with M (resp. N) contiguous (transA = 1, resp. transB = 0)
 // SINGLE: the GEMM has one K-slice, so the half-tile's block is already the final value of C there
 // A_BIG / B_BIG: the operand has a tensor map with double-size boxes (one TMA operation per 128 rows or columns)
@@ -92,7 +101,7 @@ struct cleave_plan_s {
 
     // exec work list: tiles of the original tasks in raster order, then each reissue's tiles
     std::vector<cleave::TileDesc> tiles;
-    std::vector<uint32_t> task_ntiles;             // per task: number of half-tiles
+    std::vector<uint32_t> task_ntiles;             // per task: number of (half-tile, segment) quadrants
     // in-kernel K-slice sum: cell c (one half-tile position of a GEMM with several K-slices) owns the
     // ksplit[gemm] consecutive entries of fin_refs starting at fin_ref0[c], slice order
     std::vector<uint32_t> fin_ref0;

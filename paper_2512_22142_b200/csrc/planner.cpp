@@ -492,11 +492,16 @@ int plan_reissue(cleave_plan_s& p, const uint32_t* failed, uint32_t n, uint32_t*
 }
 
 // ---- exec work list -----------------------------------------------------------------------------
-// A task is cut into half-tiles of 128 rows x <= 256 columns; two half-tiles with the same GEMM,
-// K-range and columns form a pair, the unit a cluster of two CTAs runs (one CTA per half).  The
-// halves of a pair need not be neighbours nor belong to the same task: in a column strip every
-// block has the same columns, so a block of an odd number of 128-row granules shares a pair with
-// the block below it and no MMA rows stay empty.
+// The exec kernel's unit is a pair of half-tiles (128 rows x <= 256 columns each, same GEMM, K-range
+// and columns; one CTA of a cluster per half).  Two ways to cut a GEMM into pairs:
+//
+//   grid      All block edges of the GEMM's tasks lie on multiples of 128 (the default granules): the
+//             GEMM is cut, K-range by K-range, on a global grid of 256 x 256 pairs, whatever the
+//             blocks' shapes.  Each 128 x 128 quadrant of a pair is the cell of whichever task owns it
+//             there and is stored into that task's block, so narrow, short or odd-sized blocks cost
+//             no tensor-core work: every pair is full except at the GEMM's edges.
+//   per task  Otherwise (and for replacement tasks) every task is cut into half-tiles of its own,
+//             <= 256 columns wide, and half-tiles with equal GEMM, K-range and columns share a pair.
 //
 // Order of the pairs (tiles running at the same time share operand panels in L2): by DAG level,
 // GEMM, K-range, band of 4096 rows, column, row.  (Walking a GEMM cell by cell, all K-slices of a
@@ -514,6 +519,96 @@ struct Half {
     uint32_t kslice;
 };
 
+TileSeg no_seg(uint32_t task) {
+    TileSeg s;
+    s.task = task; s.ld = 0; s.out_off = 0; s.fin = kNoFin; s.live = 0;
+    return s;
+}
+
+TileDesc tile_header(const cleave_plan_s& p, uint32_t gi, uint32_t k0, uint32_t k1, uint32_t kslice, uint32_t n_col, uint32_t cols,
+                     uint32_t split) {
+    const cleave_gemm_t& g = p.gemms[gi];
+    TileDesc d;
+    std::memset(&d, 0, sizeof d);
+    d.gemm = gi;
+    d.flags = (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN) | (p.ksplit[gi] == 1 ? TILE_SINGLE : 0u) |
+              ((!g.transA || g.M % 64 == 0) ? TILE_A_BIG : 0u) | ((g.transB || g.N % 64 == 0) ? TILE_B_BIG : 0u);
+    d.n_col = n_col;
+    d.n_mma = ((cols + 15) / 16 * 16) | (cols << 16);
+    d.k0 = k0; d.k1 = k1;
+    d.ldc = g.N;
+    d.level = (uint32_t)g.level | (std::min(p.ksplit[gi], 255u) << 16) | (std::min(kslice, 255u) << 24);
+    d.split = split;
+    return d;
+}
+
+// Grid tiling of GEMM gi over its original tasks `ids`.  Returns false (nothing appended) when the
+// GEMM does not qualify.
+bool grid_tiles(cleave_plan_s& p, uint32_t gi, const std::vector<uint32_t>& ids) {
+    const cleave_gemm_t& g = p.gemms[gi];
+    const uint32_t S = p.ksplit[gi];
+    const uint32_t Mc = (uint32_t)cdiv(g.M, 128), Nc = (uint32_t)cdiv(g.N, 128);
+    if ((uint64_t)Mc * Nc * S > (1ull << 26)) return false;
+    std::vector<uint32_t> owner((size_t)Mc * Nc * S, UINT32_MAX);
+    std::vector<uint32_t> sk0(S, UINT32_MAX), sk1(S, 0);
+    for (uint32_t id : ids) {
+        const cleave_task_t& t = p.tasks[id];
+        if (t.m0 % 128 || t.n0 % 128 || (t.m1 % 128 && t.m1 != g.M) || (t.n1 % 128 && t.n1 != g.N) || t.kslice >= S) return false;
+        if (sk0[t.kslice] == UINT32_MAX) { sk0[t.kslice] = t.k0; sk1[t.kslice] = t.k1; }
+        else if (sk0[t.kslice] != t.k0 || sk1[t.kslice] != t.k1) return false;      // one K-range per slice
+        for (uint32_t r = t.m0 / 128; r < cdiv(t.m1, 128); ++r)
+            for (uint32_t c = t.n0 / 128; c < cdiv(t.n1, 128); ++c) {
+                uint32_t& o = owner[((size_t)t.kslice * Mc + r) * Nc + c];
+                if (o != UINT32_MAX) return false;
+                o = id;
+            }
+    }
+    for (uint32_t o : owner) if (o == UINT32_MAX) return false;
+    // cells of the in-kernel K-slice sum: one per 128 x 128 quadrant, the same in every slice
+    const bool fin = S >= 2 && S <= 8 && g.N % 4 == 0;
+    uint32_t cell0 = 0;
+    if (fin) {
+        p.gemm_finishable[gi] = 1;
+        cell0 = (uint32_t)p.fin_ref0.size();
+        for (uint32_t r = 0; r < Mc; ++r)
+            for (uint32_t c = 0; c < Nc; ++c) {
+                p.fin_ref0.push_back((uint32_t)p.fin_refs.size());
+                for (uint32_t s = 0; s < S; ++s) {
+                    const cleave_task_t& t = p.tasks[owner[((size_t)s * Mc + r) * Nc + c]];
+                    const uint32_t ld = t.n1 - t.n0;
+                    p.fin_refs.push_back(FinRef{t.part_off + (uint64_t)(r * 128 - t.m0) * ld + (c * 128 - t.n0), ld, t.id});
+                }
+            }
+    }
+    for (uint32_t s = 0; s < S; ++s)
+        for (uint32_t tj = 0; tj < cdiv(Nc, 2); ++tj)
+            for (uint32_t ti = 0; ti < cdiv(Mc, 2); ++ti) {
+                const uint32_t n_col = tj * 256, cols = std::min(256u, g.N - n_col);
+                const uint32_t nseg = cols > 128 ? 2u : 1u;
+                TileDesc d = tile_header(p, gi, sk0[s], sk1[s], s, n_col, cols, nseg == 2 ? 128u : cols);
+                for (uint32_t r = 0; r < 2; ++r) {
+                    const uint32_t cr = 2 * ti + r;
+                    TileHalf& h = d.h[r];
+                    h.m_row = cr * 128;
+                    h.rows = cr < Mc ? std::min(128u, g.M - cr * 128) : 0u;
+                    for (uint32_t q = 0; q < 2; ++q) {
+                        const uint32_t cc = 2 * tj + q;
+                        if (!h.rows || q >= nseg) { h.seg[q] = no_seg(0); continue; }
+                        const cleave_task_t& t = p.tasks[owner[((size_t)s * Mc + cr) * Nc + cc]];
+                        TileSeg& sg = h.seg[q];
+                        sg.task = t.id;
+                        sg.ld = t.n1 - t.n0;
+                        sg.out_off = t.part_off + (uint64_t)(h.m_row - t.m0) * sg.ld + (cc * 128 - t.n0);
+                        sg.fin = fin ? cell0 + cr * Nc + cc : kNoFin;
+                        sg.live = 0;
+                        p.task_ntiles[t.id] += 1;
+                    }
+                }
+                p.tiles.push_back(d);
+            }
+    return true;
+}
+
 // widths of the column tiles of a block of beta columns
 void column_tiles(uint32_t beta, std::vector<uint32_t>& w) {
     w.clear();
@@ -522,58 +617,43 @@ void column_tiles(uint32_t beta, std::vector<uint32_t>& w) {
     for (uint32_t j = 0; j < nt; ++j) w.push_back(std::min(256u, beta - j * 256));
 }
 
-}  // namespace
-
-void build_tiles(cleave_plan_s& p, uint32_t first_task) {
-    const uint32_t kBandRows = 4096;
-    const bool original = (first_task == 0);
-    p.task_ntiles.resize(p.tasks.size(), 0);
-    if (original) {
-        p.n_levels = 1;
-        for (const auto& g : p.gemms) p.n_levels = std::max<uint32_t>(p.n_levels, (uint32_t)g.level + 1);
-        p.gemm_finishable.assign(p.gemms.size(), 0);
-        p.fin_ref0.clear(); p.fin_refs.clear();
-    }
+// Per-task tiling of the listed tasks (all of one GEMM when `cells`: then the GEMM's cells of the
+// in-kernel K-slice sum are made here).
+void task_tiles(cleave_plan_s& p, const std::vector<uint32_t>& ids, bool cells) {
     std::vector<Half> halves;
     std::vector<uint32_t> widths;
-    for (uint32_t id = first_task; id < p.tasks.size(); ++id) {
+    for (uint32_t id : ids) {
         const cleave_task_t& t = p.tasks[id];
-        const cleave_gemm_t& g = p.gemms[t.gemm];
         const uint32_t alpha = t.m1 - t.m0, beta = t.n1 - t.n0;
-        if ((t.k0 % 64) || ((t.k1 % 64) && t.k1 != g.K) || (g.transA && (t.m0 % 8)) || (!g.transB && (t.n0 % 8)) ||
-            (g.lda % 8) || (g.ldb % 8))
-            p.exec_unsupported = 1;
         column_tiles(beta, widths);
         const uint32_t mh = (uint32_t)cdiv(alpha, 128);
-        p.task_ntiles[id] = mh * (uint32_t)widths.size();      // bookkeeping counts half-tiles
+        p.task_ntiles[id] = mh * (uint32_t)widths.size();
         for (uint32_t hi = 0; hi < mh; ++hi) {
             uint32_t col = 0;
             for (uint32_t wj : widths) {
                 Half x;
                 x.key = HalfKey{t.gemm, t.k0, t.k1, t.n0 + col, wj};
-                x.h.task = id;
                 x.h.m_row = t.m0 + hi * 128;
                 x.h.rows = std::min(128u, alpha - hi * 128);
-                x.h.ld = beta;
-                x.h.out_off = t.part_off + (uint64_t)hi * 128 * beta + col;
-                x.h.fin = kNoFin;
-                x.h.pad = 0;
+                x.h.seg[0].task = id;
+                x.h.seg[0].ld = beta;
+                x.h.seg[0].out_off = t.part_off + (uint64_t)hi * 128 * beta + col;
+                x.h.seg[0].fin = kNoFin;
+                x.h.seg[0].live = 0;
+                x.h.seg[1] = no_seg(id);
                 x.kslice = t.kslice;
                 halves.push_back(x);
                 col += wj;
             }
         }
     }
-
-    // ---- cells of the in-kernel K-slice sum (original plan only): a GEMM qualifies when every half-tile
-    // position holds exactly one half-tile per K-slice, all of equal shape, and float4 accesses are aligned
-    if (original) {
-        std::vector<std::vector<uint32_t>> by_gemm(p.gemms.size());
-        for (uint32_t i = 0; i < halves.size(); ++i) by_gemm[halves[i].key.gemm].push_back(i);
-        for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
-            const uint32_t S = p.ksplit[gi];
-            if (S < 2 || S > 8 || p.gemms[gi].N % 4) continue;
-            std::vector<uint32_t>& idx = by_gemm[gi];
+    // cells: the GEMM qualifies when every half-tile position holds exactly one half-tile per K-slice, all of
+    // equal shape, and float4 accesses are aligned
+    if (cells && !halves.empty()) {
+        const uint32_t gi = halves[0].key.gemm, S = p.ksplit[gi];
+        if (S >= 2 && S <= 8 && p.gemms[gi].N % 4 == 0) {
+            std::vector<uint32_t> idx(halves.size());
+            for (uint32_t i = 0; i < idx.size(); ++i) idx[i] = i;
             std::sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
                 const Half &x = halves[a], &y = halves[b];
                 if (x.h.m_row != y.h.m_row) return x.h.m_row < y.h.m_row;
@@ -585,24 +665,24 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
                 for (uint32_t s = 0; ok && s < S; ++s) {
                     const Half &x = halves[idx[c + s]], &x0 = halves[idx[c]];
                     ok = x.kslice == s && x.h.m_row == x0.h.m_row && x.h.rows == x0.h.rows && x.key.n_col == x0.key.n_col &&
-                         x.key.cols == x0.key.cols && x.key.n_col % 4 == 0 && x.key.cols % 4 == 0 && x.h.ld % 4 == 0 &&
-                         x.h.out_off % 4 == 0;
+                         x.key.cols == x0.key.cols && x.key.n_col % 4 == 0 && x.key.cols % 4 == 0 && x.h.seg[0].ld % 4 == 0 &&
+                         x.h.seg[0].out_off % 4 == 0;
                 }
-            if (!ok) continue;
-            p.gemm_finishable[gi] = 1;
-            for (size_t c = 0; c < idx.size(); c += S) {
-                const uint32_t cell = (uint32_t)p.fin_ref0.size();
-                p.fin_ref0.push_back((uint32_t)p.fin_refs.size());
-                for (uint32_t s = 0; s < S; ++s) {
-                    Half& x = halves[idx[c + s]];
-                    x.h.fin = cell;
-                    p.fin_refs.push_back(FinRef{x.h.out_off, x.h.ld, x.h.task});
+            if (ok) {
+                p.gemm_finishable[gi] = 1;
+                for (size_t c = 0; c < idx.size(); c += S) {
+                    const uint32_t cell = (uint32_t)p.fin_ref0.size();
+                    p.fin_ref0.push_back((uint32_t)p.fin_refs.size());
+                    for (uint32_t s = 0; s < S; ++s) {
+                        Half& x = halves[idx[c + s]];
+                        x.h.seg[0].fin = cell;
+                        p.fin_refs.push_back(FinRef{x.h.seg[0].out_off, x.h.seg[0].ld, x.h.seg[0].task});
+                    }
                 }
             }
         }
     }
-
-    // ---- pairs: consecutive half-tiles (by row) of the same GEMM, K-range and columns
+    // pairs: consecutive half-tiles (by row) of the same GEMM, K-range and columns
     std::stable_sort(halves.begin(), halves.end(), [](const Half& a, const Half& b) {
         if (a.key.gemm != b.key.gemm) return a.key.gemm < b.key.gemm;
         if (a.key.k0 != b.key.k0) return a.key.k0 < b.key.k0;
@@ -611,25 +691,50 @@ void build_tiles(cleave_plan_s& p, uint32_t first_task) {
         if (a.key.cols != b.key.cols) return a.key.cols < b.key.cols;
         return a.h.m_row < b.h.m_row;
     });
-    const size_t begin = p.tiles.size();
     for (size_t i = 0; i < halves.size();) {
         const Half& x = halves[i];
-        const cleave_gemm_t& g = p.gemms[x.key.gemm];
-        TileDesc d;
-        std::memset(&d, 0, sizeof d);
-        d.gemm = x.key.gemm;
-        d.flags = (g.transA ? TILE_A_MN : 0u) | (g.transB ? 0u : TILE_B_MN) | (p.ksplit[d.gemm] == 1 ? TILE_SINGLE : 0u) |
-                  ((!g.transA || g.M % 64 == 0) ? TILE_A_BIG : 0u) | ((g.transB || g.N % 64 == 0) ? TILE_B_BIG : 0u);
-        d.n_col = x.key.n_col;
-        d.n_mma = ((x.key.cols + 15) / 16 * 16) | (x.key.cols << 16);
-        d.k0 = x.key.k0; d.k1 = x.key.k1;
-        d.ldc = g.N;
-        d.level = (uint32_t)g.level | (std::min(p.ksplit[d.gemm], 255u) << 16) | (std::min(x.kslice, 255u) << 24);
+        TileDesc d = tile_header(p, x.key.gemm, x.key.k0, x.key.k1, x.kslice, x.key.n_col, x.key.cols, x.key.cols);
         d.h[0] = x.h;
         // each CTA of the pair loads, multiplies and stores its own half, so any two half-tiles may share a pair
         if (i + 1 < halves.size() && halves[i + 1].key == x.key) { d.h[1] = halves[i + 1].h; i += 2; }
-        else { d.h[1].task = x.h.task; d.h[1].fin = kNoFin; i += 1; }
+        else { d.h[1].m_row = 0; d.h[1].rows = 0; d.h[1].seg[0] = d.h[1].seg[1] = no_seg(x.h.seg[0].task); i += 1; }
         p.tiles.push_back(d);
+    }
+}
+
+}  // namespace
+
+void build_tiles(cleave_plan_s& p, uint32_t first_task) {
+    const uint32_t kBandRows = 4096;
+    const bool original = (first_task == 0);
+    const size_t begin = p.tiles.size();
+    p.task_ntiles.resize(p.tasks.size(), 0);
+    if (original) {
+        p.n_levels = 1;
+        for (const auto& g : p.gemms) p.n_levels = std::max<uint32_t>(p.n_levels, (uint32_t)g.level + 1);
+        p.gemm_finishable.assign(p.gemms.size(), 0);
+        p.fin_ref0.clear(); p.fin_refs.clear();
+    }
+    std::vector<std::vector<uint32_t>> by_gemm(p.gemms.size());
+    for (uint32_t id = first_task; id < p.tasks.size(); ++id) {
+        const cleave_task_t& t = p.tasks[id];
+        const cleave_gemm_t& g = p.gemms[t.gemm];
+        if ((t.k0 % 64) || ((t.k1 % 64) && t.k1 != g.K) || (g.transA && (t.m0 % 8)) || (!g.transB && (t.n0 % 8)) ||
+            (g.lda % 8) || (g.ldb % 8))
+            p.exec_unsupported = 1;
+        by_gemm[t.gemm].push_back(id);
+    }
+    for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
+        if (by_gemm[gi].empty()) continue;
+        if (original) {
+            const size_t tiles0 = p.tiles.size(), ref0 = p.fin_ref0.size(), refs0 = p.fin_refs.size();
+            if (grid_tiles(p, gi, by_gemm[gi])) continue;
+            // not on the 128-grid: undo whatever the attempt counted, cut task by task
+            p.tiles.resize(tiles0); p.fin_ref0.resize(ref0); p.fin_refs.resize(refs0);
+            p.gemm_finishable[gi] = 0;
+            for (uint32_t id : by_gemm[gi]) p.task_ntiles[id] = 0;
+        }
+        task_tiles(p, by_gemm[gi], original);
     }
     std::stable_sort(p.tiles.begin() + begin, p.tiles.end(), [&](const TileDesc& a, const TileDesc& b) {
         const uint32_t la = a.level & 0xFFFFu, lb = b.level & 0xFFFFu;

@@ -44,13 +44,16 @@ def test_in_kernel_sum_of_k_split_cells_is_bit_identical(opts):
 
 
 def test_unequal_slices_fall_back_to_the_assembly_kernel():
-    """Memory budgets so small that the K-slices of a block are repaired into different pieces: such a
-    GEMM cannot be summed cell by cell in the exec kernel and goes through cleave_assemble; the
-    result is the same."""
+    """Blocks off the 128-grid (granule 64) under memory budgets so small that the K-slices of a block
+    are repaired into different pieces: such a GEMM cannot be summed cell by cell in the exec kernel
+    and goes through cleave_assemble; the result is the same.  (On the 128-grid the kernel's cells do
+    not depend on the blocks' shapes: the same budgets with granule 128 need no assembly kernel.)"""
     gemms, tensors = ci.projection_gemms(512, [("p", 512, 384)], ("fwd", "wgrad"))
     w = ci.Workload("tight", gemms, tensors, n_devices=12, mem_range=(150_000, 3_000_000), seed=0)
     ts = ci.make_tensors(w, integer=True)
-    opts = dict(kslice_max=128, gran_m=128, gran_n=128, gran_k=64)
+    on_grid = lib_plan_for(w, kslice_max=128, gran_m=128, gran_n=128, gran_k=64)
+    assert on_grid.finishable(0) and on_grid.finishable(1)
+    opts = dict(kslice_max=128, gran_m=64, gran_n=64, gran_k=64)
     p, op = lib_plan_for(w, **opts), oracle_plan_for(w, **opts)
     assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
     assert p.ksplit(0) == 4 and not p.finishable(0) and not p.finishable(1)
