@@ -35,18 +35,21 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 def measured_traffic(kernel: str):
-    """DRAM bytes per full-size launch recorded from an ncu capture (profiles/dram_traffic.txt), or
-    None when there is no record or the kernel's source changed since the counters were taken."""
+    """(DRAM bytes per full-size launch, how they were obtained) from the ncu record in
+    profiles/dram_traffic.txt, or (None, reason) when there is no record or the kernel's source
+    changed since the counters were taken."""
     import hashlib
     try:
         with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
             rec = json.load(f)[kernel]
         with open(os.path.join(ROOT, rec["source"]), "rb") as f:
-            if hashlib.sha1(f.read()).hexdigest() != rec["sha1"] or rec["dram_bytes_half_size_launch"] is None:
-                return None
-        return rec["dram_bytes_half_size_launch"] * rec["scale_to_full"]
+            if hashlib.sha1(f.read()).hexdigest() != rec["sha1"]:
+                return None, "kernel source changed since the capture"
+        if rec.get("dram_bytes_captured_launch") is None:
+            return None, "no capture recorded"
+        return rec["dram_bytes_captured_launch"] * rec["scale_to_full"], rec["how"]
     except Exception:
-        return None
+        return None, "no capture recorded"
 
 
 def load_peaks():
@@ -234,6 +237,79 @@ def job_throughput(flop_per_replica: float, world: int, ms_per_step: float) -> f
 
 
 # --------------------------------------------------------------------------------------------------
+# a short leg on another workload or mode (reported under config.other_workloads)
+# --------------------------------------------------------------------------------------------------
+def plan_summary(plan, n_gemms, n_devices):
+    """The paper's quantities of a plan: modelled makespans against the water-fill level, devices with work."""
+    import numpy as np
+    t = plan.tasks()
+    ratios = [plan.makespan_ns(i) / plan.tstar_ns(i) for i in range(n_gemms) if plan.tstar_ns(i)]
+    return {"tasks": int(plan.num_tasks), "tiles": int(plan.num_tiles),
+            "active_devices": int(len(np.unique(t["dev"]))) if n_devices else None,
+            "makespan_over_waterfill_level_median": float(np.median(ratios)) if ratios else None,
+            "modelled_step_makespan_ms": plan.step_makespan_ns / 1e6}
+
+
+def quick_leg(cl, ci, torch, dev, name, cfg, scale, opts, mode, min_s=0.6, tensors=None, bf16_out=False):
+    """Plans the workload, runs it for at least `min_s` seconds untimed, then times the same number of
+    steps again: step / exec / assembly times from CUDA events on the launching stream."""
+    w = ci.config(cfg, scale)
+    if tensors is None:
+        tensors = {k: t.to(dev) for k, t in ci.make_tensors(w).items()}
+    devs = ci.workload_devices(w)
+    o = cl.default_opts(**opts)
+    plan = cl.plan_uniform(w.gemms, *w.uniform, o) if devs is None else cl.plan(w.gemms, devs, o)
+    A = [tensors[g.a_key] for g in w.gemms]
+    B = [tensors[g.b_key] for g in w.gemms]
+    partials = torch.empty(max(1, plan.arena_elems), dtype=torch.float32, device=dev)
+    C = [torch.empty((g.M, g.N), dtype=torch.bfloat16 if bf16_out else torch.float32, device=dev) for g in w.gemms]
+
+    def step():
+        if mode == "two-step":
+            plan.exec_opts(A, B, partials, C, bf16=bf16_out)
+        else:
+            plan.exec_opts(A, B, partials, C, direct=True, finish=True, bf16=bf16_out)
+        plan.assemble(partials, C)
+
+    n, t0 = 0, time.perf_counter()
+    while True:
+        step(); n += 1
+        if n % 8 == 0:
+            torch.cuda.synchronize()
+            if time.perf_counter() - t0 >= min_s:
+                break
+    plan.check_status()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n)]
+    torch.cuda.synchronize()
+    for e in ev:
+        e[0].record()
+        if mode == "two-step":
+            plan.exec_opts(A, B, partials, C, bf16=bf16_out)
+        else:
+            plan.exec_opts(A, B, partials, C, direct=True, finish=True, bf16=bf16_out)
+        e[1].record()
+        plan.assemble(partials, C)
+        e[2].record()
+    torch.cuda.synchronize()
+    plan.check_status()
+    step_ms = ev[0][0].elapsed_time(ev[-1][2]) / n
+    exec_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    asm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    S = [plan.ksplit(i) for i in range(len(w.gemms))]
+    asm_bytes = float(sum((S[i] + 1) * g.M * g.N * 4 for i, g in enumerate(w.gemms)
+                          if mode == "two-step" or not (S[i] == 1 or plan.finishable(i))))
+    out = {"name": name, "workload": w.name, "opts": opts, "write_out": mode, "c_dtype": "bf16" if bf16_out else "fp32",
+           "steps_timed": n, "step_ms": step_ms, "step_TFLOPs": w.flops / step_ms / 1e9, "exec_ms": exec_ms,
+           "exec_TFLOPs": w.flops / exec_ms / 1e9, "assemble_ms": asm_ms,
+           "assemble_GBs": asm_bytes / asm_ms / 1e6 if asm_bytes else None, "assemble_bytes": asm_bytes,
+           "arena_GB": plan.arena_elems * 4 / 1e9, "ksplit_max": max(S)}
+    out.update(plan_summary(plan, len(w.gemms), w.n_devices))
+    plan.close()
+    del partials, C
+    return out
+
+
+# --------------------------------------------------------------------------------------------------
 # the CUDA path
 # --------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -269,14 +345,17 @@ def run_ours(args):
     gen_s = time.perf_counter() - t0
     devs = ci.workload_devices(w)
     t0 = time.perf_counter()
-    plan = cl.plan_uniform(w.gemms, *w.uniform, cl.default_opts(**opts)) if devs is None else cl.plan(w.gemms, devs, cl.default_opts(**opts))
+    plan_opts = cl.default_opts(**opts)
+    plan = cl.plan_uniform(w.gemms, *w.uniform, plan_opts) if devs is None else cl.plan(w.gemms, devs, plan_opts)
     plan_ms = (time.perf_counter() - t0) * 1e3
 
     d_tensors = {k: t.to(dev) for k, t in tensors.items()}
     A = [d_tensors[g.a_key] for g in w.gemms]
     B = [d_tensors[g.b_key] for g in w.gemms]
     partials = torch.empty(plan.arena_elems, dtype=torch.float32, device=dev)
-    C = [torch.empty((g.M, g.N), dtype=torch.float32, device=dev) for g in w.gemms]
+    c_dtype = torch.bfloat16 if args.bf16_out else torch.float32
+    c_bytes = 2 if args.bf16_out else 4
+    C = [torch.empty((g.M, g.N), dtype=c_dtype, device=dev) for g in w.gemms]
     flops = float(w.flops)
     S = [plan.ksplit(i) for i in range(len(w.gemms))]
     # bytes the assembly kernels move: GEMMs with one K-slice are finished by the exec kernel in fused mode
@@ -295,13 +374,19 @@ def run_ours(args):
     def run_exec():
         # one-slice GEMMs are written straight to C by the exec kernel unless --two-step is given
         if args.two_step:
-            plan.exec(A, B, partials)
+            plan.exec_opts(A, B, partials, C, bf16=args.bf16_out)
         else:
-            plan.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish)
+            plan.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish, bf16=args.bf16_out)
 
-    for _ in range(args.warmup):
+    # warm-up: at least --warmup steps AND at least --min-warm-s seconds of back-to-back steps, so that the
+    # timed steps see the clocks of a long run (the power cap pulls them down within about a second)
+    warm_steps, t_warm = 0, time.perf_counter()
+    while warm_steps < args.warmup or time.perf_counter() - t_warm < args.min_warm_s:
         run_exec()
         plan.assemble(partials, C)
+        warm_steps += 1
+        if warm_steps % 8 == 0:
+            torch.cuda.synchronize()
     plan.check_status()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     sampler = ClockSampler(local) if rank == 0 else None
@@ -328,10 +413,10 @@ def run_ours(args):
     value = job_throughput(flops, world, ms_per_step)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----------------
-    host_C = [torch.empty((g.M, g.N), dtype=torch.float32).pin_memory() if args.e2e_steps > 0 else
-              torch.empty((g.M, g.N), dtype=torch.float32) for g in w.gemms]
+    host_C = [torch.empty((g.M, g.N), dtype=c_dtype).pin_memory() if args.e2e_steps > 0 else
+              torch.empty((g.M, g.N), dtype=c_dtype) for g in w.gemms]
     h2d = sum(t.numel() * 2 for t in tensors.values())
-    d2h = sum(c.numel() * 4 for c in host_C)
+    d2h = sum(c.numel() * c_bytes for c in host_C)
 
     def e2e_step():
         for k, t in tensors.items():
@@ -384,9 +469,9 @@ def run_ours(args):
                     s_comp.wait_event(out_done[i - 2])           # this output set has been copied out
                 Ai, Bi = [dt[g.a_key] for g in w.gemms], [dt[g.b_key] for g in w.gemms]
                 if args.two_step:
-                    pl.exec(Ai, Bi, partials)
+                    pl.exec_opts(Ai, Bi, partials, Cs, bf16=args.bf16_out)
                 else:
-                    pl.exec_fused(Ai, Bi, partials, Cs)
+                    pl.exec_opts(Ai, Bi, partials, Cs, direct=True, finish=not args.no_finish, bf16=args.bf16_out)
                 pl.assemble(partials, Cs)
                 comp_done[i].record(s_comp)
             with torch.cuda.stream(s_out):
@@ -409,7 +494,7 @@ def run_ours(args):
         plan_b.check_status()
         e2e_ms = max_over_ranks(t_begin.elapsed_time(t_end)) / (n_pipe - 2)
     e2e_value = job_throughput(flops, world, e2e_ms)
-    checksum = float(host_C[0][0, :8].double().sum())
+    checksum = float(host_C[0][0, :8].double().sum()) if args.e2e_steps > 0 else None
 
     if rank != 0:
         if dist is not None:
@@ -423,9 +508,9 @@ def run_ours(args):
         failed = ci.make_failed_ids(p2.num_tasks, 0.10, w.seed + 2)
         p2.set_drops(failed)
         if args.two_step:
-            p2.exec(A, B, partials)
+            p2.exec_opts(A, B, partials, C, bf16=args.bf16_out)
         else:
-            p2.exec_fused(A, B, partials, C)
+            p2.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish, bf16=args.bf16_out)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         c0, c1, c2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
@@ -443,7 +528,7 @@ def run_ours(args):
 
     # ---- block verification (Section 6 of the paper), once, on the result of the last step -------------------
     verify = None
-    if not args.no_verify:
+    if not args.no_verify and not (args.bf16_out and not args.two_step):
         t = plan.tasks()
         live = (t["flags"] & 1) == 0
         al, be, ka = (t["m1"] - t["m0"]).astype(np.float64), (t["n1"] - t["n0"]).astype(np.float64), (t["k1"] - t["k0"]).astype(np.float64)
@@ -455,37 +540,91 @@ def run_ours(args):
         v1.record()
         torch.cuda.synchronize()
         vms = v0.elapsed_time(v1)
-        verify = {"flagged_tasks": int(n_bad), "ms": vms, "algorithmic_GB": vbytes / 1e9, "GB_per_s": vbytes / vms / 1e6,
-                  "frac_of_measured_hbm": vbytes / vms / 1e6 / load_peaks()[0]["hbm_gbs"]}
+        verify = {"flagged_tasks": int(n_bad), "ms": vms, "dispatch_volume_GB": vbytes / 1e9,
+                  "dispatch_volume_GB_per_s": vbytes / vms / 1e6,
+                  "note": "bytes = every task's own rows, columns and block (the method's dispatch + return volume); "
+                          "tasks share operand panels, so part of it is served by L2: a rate, not a DRAM roofline fraction"}
+
+    # ---- other modes and workloads, short legs (rank 0, N = 1): observed in the same run as the headline ----
+    others = []
+    if world == 1 and not args.no_other:
+        shared = dict(tensors=d_tensors)
+        base = dict(opts)
+        legs = [("same workload, two-step (cleave_exec + cleave_assemble of every GEMM)", args.config, args.scale, base, "two-step", False, shared),
+                ("same workload, bf16 outputs", args.config, args.scale, base, "fused", True, shared)]
+        if args.gran_m is None:
+            legs.append(("same workload, row granule 256", args.config, args.scale, dict(base, gran_m=256), "fused", False, shared))
+        if args.config == 3 and args.scale == 1:
+            legs += [("GPT-2-small-shaped layer, 64 devices", 2, 1, {}, "fused", False, {}),
+                     ("Llama-13B-shaped layer, 4096 devices", 5, 1, {}, "fused", False, {}),
+                     ("attention GEMMs of 1024 heads as tasks, 64 devices", 6, 1, {}, "fused", False, {})]
+        for name, cfg, scale, o, mode, b16, kw in legs:
+            try:
+                others.append(quick_leg(cl, ci, torch, dev, name, cfg, scale, o, mode, bf16_out=b16, **kw))
+            except Exception as e:                          # a leg must not cost the headline its line
+                others.append({"name": name, "error": repr(e)})
+            torch.cuda.empty_cache()
 
     peaks, peak_kind = load_peaks()
     exec_tflops = flops / (exec_ms * 1e-3) / 1e12
-    asm_gbs = asm_bytes / (asm_ms * 1e-3) / 1e9
+    sm_mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    flop_per_clk_per_sm = flops / (exec_ms * 1e-3) / (sm_mhz * 1e6) / sm_count if sm_mhz else None
+    traffic, traffic_how = (measured_traffic("exec_pair_kernel") if (args.config == 3 and args.scale == 1 and not args.two_step
+                                                                      and not args.bf16_out and not args.no_finish)
+                            else (None, "recorded for the default run of the Llama-7B-shaped layer only"))
+    # the assembly kernels only run where the exec kernel cannot finish a GEMM itself: their roofline comes from
+    # this run when it launches them, else from the two-step leg above
+    asm_src = {"ms": asm_ms, "bytes": asm_bytes, "from": "this run's steps"} if asm_bytes else None
+    if asm_src is None:
+        for o in others:
+            if o.get("write_out") == "two-step" and o.get("assemble_bytes"):
+                asm_src = {"ms": o["assemble_ms"], "bytes": o["assemble_bytes"], "from": "the two-step leg of this run (config.other_workloads[0])"}
+    asm_traffic, asm_traffic_how = measured_traffic("assemble_vec_kernel")
+    roofline_assemble = None
+    if asm_src:
+        asm_gbs = asm_src["bytes"] / (asm_src["ms"] * 1e-3) / 1e9
+        roofline_assemble = {"kernel": "assemble_vec_kernel", "bound": "hbm", "achieved": asm_gbs, "peak": peaks["hbm_gbs"],
+                             "unit": "GB/s", "frac": asm_gbs / peaks["hbm_gbs"],
+                             "traffic": asm_traffic if (args.config == 3 and args.scale == 1) else None, "traffic_how": asm_traffic_how,
+                             "peak_kind": f"{peak_kind} copy bandwidth", "frac_of_nominal": asm_gbs / NOMINAL_HBM_GBS,
+                             "algorithmic_bytes": asm_src["bytes"], "timed_in": asm_src["from"]}
+    step_s = warm_steps * ms_per_step * 1e-3
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm_steps,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": w.name, "gemms": len(w.gemms), "devices": w.n_devices, "tasks": plan.num_tasks,
-            "tiles": plan.num_tiles, "flop_per_step": flops, "ksplit": S, "arena_GB": plan.arena_elems * 4 / 1e9,
+            "workload": w.name, "gemms": len(w.gemms), "devices": w.n_devices, "flop_per_step": flops, "ksplit": S,
+            "granule": [plan_opts.gran_m, plan_opts.gran_n, plan_opts.gran_k], "kslice_max": plan_opts.kslice_max,
+            "plan": plan_summary(plan, len(w.gemms), w.n_devices), "arena_GB": plan.arena_elems * 4 / 1e9,
             "parallelism": "replicas only" if world > 1 else "1 GPU",
-            "write_out": "two-step" if args.two_step else "fused for one-slice GEMMs",
+            "write_out": ("two-step: every block to the arena, every GEMM through cleave_assemble" if args.two_step else
+                          "in the exec kernel: one-slice blocks stored in C" +
+                          ("" if args.no_finish else ", K-split cells summed in fixed order by the block stored last")),
+            "c_dtype": "bf16" if args.bf16_out else "fp32",
+            "gemms_finished_in_exec_kernel": int(sum(in_kernel)),
             "l2": "not flushed; operands + arena + outputs per step (~%.1f GB) far exceed the 126 MB L2" %
                   ((h2d + plan.arena_elems * 4 + d2h) / 1e9),
-            "plan_ms_host": plan_ms, "step_ms_median": statistics.median(step_times), "step_ms_best": min(step_times), "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
+            "warmup": f"{warm_steps} steps, about {step_s:.1f} s back to back (at least --warmup steps and --min-warm-s seconds)",
+            "plan_ms_host": plan_ms, "step_ms_median": statistics.median(step_times), "step_ms_best": min(step_times),
+            "input_gen_s": gen_s, "exec_ms": exec_ms, "assemble_ms": asm_ms,
             "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
             "pct_of_measured_sustained_bf16": 100 * value / world / peaks["bf16_tflops_sustained"],
             "churn": churn, "verify": verify, "e2e_ms_per_step": e2e_ms, "e2e_serial_ms_per_step": e2e_serial_ms,
-            "e2e_mode": "pipelined over 3 streams, 2 buffer sets; every step copies all inputs in and all results out", "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
+            "e2e_mode": "pipelined over 3 streams, 2 buffer sets; every step copies all inputs in and all results out",
+            "e2e_steps": args.e2e_steps, "e2e_checksum": checksum,
+            "other_workloads": others,
         },
         "roofline": {"kernel": "exec_pair_kernel", "bound": "tensor", "achieved": exec_tflops, "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": exec_tflops / peaks["bf16_tflops_sustained"],
-                     "traffic": measured_traffic("exec_pair_kernel") if (args.config == 3 and args.scale == 1 and not args.two_step) else None,
-                     "peak_kind": f"{peak_kind}, sustained cuBLAS bf16 (kernel timed inside a long step)",
-                     "frac_of_burst": exec_tflops / peaks["bf16_tflops"], "frac_of_nominal": exec_tflops / NOMINAL_BF16_TFLOPS},
-        "roofline_assemble": {"kernel": "assemble_vec_kernel", "bound": "hbm", "achieved": asm_gbs, "peak": peaks["hbm_gbs"],
-                              "unit": "GB/s", "frac": asm_gbs / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind,
-                              "frac_of_nominal": asm_gbs / NOMINAL_HBM_GBS, "algorithmic_bytes": asm_bytes},
+                     "traffic": traffic, "traffic_how": traffic_how,
+                     "peak_kind": f"{peak_kind}, sustained cuBLAS bf16: the kernel is timed inside steps that follow "
+                                  f"{step_s:.1f} s of back-to-back steps (power-capped steady state)",
+                     "frac_of_burst": exec_tflops / peaks["bf16_tflops"], "frac_of_nominal": exec_tflops / NOMINAL_BF16_TFLOPS,
+                     "flop_per_clk_per_sm": flop_per_clk_per_sm,
+                     "frac_of_tensor_peak_per_clk": flop_per_clk_per_sm / 8192.0 if flop_per_clk_per_sm else None},
+        "roofline_assemble": roofline_assemble,
         "e2e": {"value": e2e_value if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": plan.num_launches * args.steps,
         "clocks": clocks,
@@ -514,6 +653,9 @@ def main():
     ap.add_argument("--two-step", action="store_true", help="cleave_exec + full cleave_assemble instead of the fused write-out")
     ap.add_argument("--no-finish", action="store_true", help="fused write-out of one-slice GEMMs only; K-split GEMMs go through cleave_assemble")
     ap.add_argument("--gran-m", type=int, default=None, help="row granule of the planner (default 128)")
+    ap.add_argument("--bf16-out", action="store_true", help="C in bf16 (rounded from the fp32 sums) instead of fp32")
+    ap.add_argument("--min-warm-s", type=float, default=1.5, help="warm up for at least this long before the timed steps")
+    ap.add_argument("--no-other", action="store_true", help="skip the short legs on other modes and workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -7,7 +7,8 @@ algorithm.  This file is a deterministic integer heuristic for the same problem,
 K-split (each output block may be cut into S K-slices whose partial blocks are summed at the
 parameter server; S = 1 is the paper's formulation).  Steps:
 
-  1  granule counts; choice of S and the nominal slice depth kappa_hat
+  1  granule counts; choice of S (deep contractions are cut; K is also cut when the GEMM's whole
+     level has fewer output cells than there are devices) and the nominal slice depth kappa_hat
   2  capacity a_k(T): largest output area device k can finish within T under each cost term and
      the memory constraint; devices that cannot take one granule cell stay idle (zero-task rule)
   3  T* = least T with sum_k a_k(T) >= S*M*N  (work proportional to capability)
@@ -50,6 +51,7 @@ class Gemm:
     K: int
     transA: int = 0
     transB: int = 0
+    level: int = 0      # DAG level (Section 4.1): GEMMs of one level are independent and run in parallel
 
 
 @dataclass(frozen=True)
@@ -176,22 +178,30 @@ def split_counts(total: int, parts: int) -> List[int]:
 # ---------------------------------------------------------------------------------- one GEMM
 
 
-def choose_ksplit(g: Gemm, n_dev: int, o: Opts, Mg: int, Ng: int, Kg: int) -> int:
+def choose_ksplit(g: Gemm, n_dev: int, o: Opts, level_cells: int, Kg: int) -> int:
+    """`level_cells`: output cells of all GEMMs of this GEMM's level together.  The GEMMs of a level
+    run in parallel over the same devices (Section 4.1), so devices are only left without a cell,
+    and K is only split to give them work, when the whole level has fewer cells than devices."""
     if o.ksplit:
         return max(1, min(o.ksplit, Kg))
     s_depth = ceil_div(g.K, o.kslice_max) if o.kslice_max else 1
-    s_fan = ceil_div(n_dev, Mg * Ng)     # more devices than output cells: split K so all can work
+    s_fan = ceil_div(n_dev, level_cells)
     return max(1, min(max(s_depth, s_fan), o.ksplit_cap, Kg))
 
 
-def plan_rectangles(g: Gemm, devices: Sequence[Device], o: Opts):
-    """Steps 1-6 for one GEMM.  Returns (S, T*, [(m0,m1,n0,n1,k0,k1,kslice,dev), ...])."""
+def output_cells(g: Gemm, o: Opts) -> int:
+    return ceil_div(g.M, o.gran_m) * ceil_div(g.N, o.gran_n)
+
+
+def plan_rectangles(g: Gemm, devices: Sequence[Device], o: Opts, level_cells: Optional[int] = None):
+    """Steps 1-6 for one GEMM.  Returns (S, T*, [(m0,m1,n0,n1,k0,k1,kslice,dev), ...]).
+    `level_cells` defaults to the GEMM's own cells (a level of its own)."""
     if g.M <= 0 or g.N <= 0 or g.K <= 0:
         raise PlanError("E_INVAL", "empty GEMM")
     if not devices:
         raise PlanError("E_NO_DEVICES")
     Mg, Ng, Kg = ceil_div(g.M, o.gran_m), ceil_div(g.N, o.gran_n), ceil_div(g.K, o.gran_k)
-    S = choose_ksplit(g, len(devices), o, Mg, Ng, Kg)
+    S = choose_ksplit(g, len(devices), o, Mg * Ng if level_cells is None else level_cells, Kg)
     s_limit = S if o.ksplit else min(o.ksplit_cap, Kg)
 
     while True:
@@ -299,8 +309,12 @@ def plan(gemms: Sequence[Gemm], devices: Sequence[Device], opts: Opts = Opts()) 
     again, Section 3.2)."""
     p = Plan(list(gemms), list(devices), opts)
     per_gemm = []
+    cells = {}
     for g in gemms:
-        S, t_star, rects = plan_rectangles(g, devices, opts)
+        if g.M > 0 and g.N > 0:
+            cells[g.level] = cells.get(g.level, 0) + output_cells(g, opts)
+    for g in gemms:
+        S, t_star, rects = plan_rectangles(g, devices, opts, cells.get(g.level))
         p.ksplit.append(S)
         p.t_star.append(t_star)
         per_gemm.append(rects)

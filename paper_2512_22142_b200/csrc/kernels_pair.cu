@@ -240,59 +240,93 @@ __device__ __forceinline__ void finish_strip(const FinRef* __restrict__ refs, ui
     }
 }
 
-// One 32 x 32 chunk of a strip whose cell is complete but for this block: the staged accumulator
-// values (own K-slice `mine`) go to the block in the arena as always, and, added to the other slices'
-// values in the fixed tree order, to C.  Lanes: 8 per row segment of 32 columns, 4 rows per step.
+// One 32 x 32 chunk of a strip whose cell is complete but for this block: the accumulator values
+// (own K-slice `mine`) go to the block in the arena as always, and, added to the other slices' values
+// in the fixed tree order, to C.  Lanes: 8 per row segment of 32 columns, 4 rows per step.  The other
+// slices' values are asked for before the accumulator chunk is read from tensor memory and staged,
+// so their latency (L2: they were prefetched when the tile was handed out) overlaps that work.
+struct SummedChunk {
+    const FinRef* refs;         // the cell's blocks, slice order
+    uint32_t nslices, mine;
+    const float* partials;
+    float* own_blk;             // the quadrant's (row0, 0) in this task's block
+    uint32_t own_ld;
+    uint32_t row0, rows_here;
+    uint32_t c0, cols;          // first column of the chunk inside the quadrant; the quadrant's columns
+    void* c_base;
+    uint64_t c_off;             // the quadrant's (0, 0) in C
+    uint32_t ldc;
+    uint32_t taddr;             // tensor-memory address of the chunk
+    bool last_chunk;            // reading it frees the accumulator slot
+    uint32_t acc_empty_leader;
+};
 template <int SP, bool BF16>
-__device__ __forceinline__ void store_chunk_summed(const float* stage_tile, const FinRef* __restrict__ refs, uint32_t nslices,
-                                                   uint32_t mine, const float* __restrict__ partials, float* own_blk,
-                                                   uint32_t own_ld, uint32_t row0, uint32_t rows_here, uint32_t c0, uint32_t cols,
-                                                   void* c_base, uint64_t c_off, uint32_t ldc, uint32_t lane) {
-    // own_blk: the quadrant's (row0, 0) in this task's block; c0: first column of the chunk inside the quadrant;
-    // cols: the quadrant's columns; c_off: offset of the quadrant's (0, 0) in C
-    constexpr int RB = SP <= 2 ? 4 : (SP <= 4 ? 2 : 1);      // rows per lane whose loads are in flight together
+__device__ __forceinline__ void summed_chunk(const SummedChunk& k, float* stage_tile, uint32_t lane) {
+    constexpr int RB = SP <= 2 ? 8 : (SP <= 4 ? 4 : 2);      // rows per lane whose loads are in flight together
+    constexpr int NO = SP - 1;                               // other slices (slot j holds slice j, or j + 1 from `mine` on)
     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
-    if (c0 + cc >= cols) rows_here = 0;                      // ragged last chunk (columns come in fours)
-    const float* src[SP];
-    uint32_t ld[SP];
+    const uint32_t rows_here = (k.c0 + cc >= k.cols) ? 0u : k.rows_here;   // ragged last chunk (columns come in fours)
+    const float* src[NO];
+    uint32_t ld[NO];
 #pragma unroll
-    for (int s = 0; s < SP; ++s) {
-        if ((uint32_t)s < nslices && (uint32_t)s != mine) { const FinRef rf = refs[s]; src[s] = partials + rf.off + (uint64_t)row0 * rf.ld + c0 + cc; ld[s] = rf.ld; }
-        else { src[s] = nullptr; ld[s] = 0; }
+    for (int j = 0; j < NO; ++j) {
+        const uint32_t s = (uint32_t)j < k.mine ? (uint32_t)j : (uint32_t)j + 1u;
+        if (s < k.nslices) { const FinRef rf = k.refs[s]; src[j] = k.partials + rf.off + (uint64_t)k.row0 * rf.ld + k.c0 + cc; ld[j] = rf.ld; }
+        else { src[j] = nullptr; ld[j] = 0; }
     }
-#pragma unroll
-    for (int b = 0; b < 8; b += RB) {
-        float4 v[RB][SP];
+    float4 o[RB][NO];
+    auto load_batch = [&](int b) {
 #pragma unroll
         for (int x = 0; x < RB; ++x) {
             const uint32_t r = rr + 4u * (uint32_t)(b + x);
 #pragma unroll
-            for (int s = 0; s < SP; ++s) {
-                v[x][s] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (r < rows_here && src[s]) v[x][s] = ld_cg_f4(src[s] + (uint64_t)r * ld[s]);
+            for (int j = 0; j < NO; ++j) {
+                o[x][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < rows_here && src[j]) o[x][j] = ld_cg_f4(src[j] + (uint64_t)r * ld[j]);
             }
         }
+    };
+    load_batch(0);
+    {
+        uint32_t v[32];
+        tmem_ld_32x32(k.taddr, v);
+        tmem_ld_wait();
+        if (k.last_chunk) {                                  // slot fully read: hand it back to the leader
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(k.acc_empty_leader);
+        }
+#pragma unroll
+        for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
+    }
+    __syncwarp();
+#pragma unroll
+    for (int b = 0; b < 8; b += RB) {
+        if (b) load_batch(b);
 #pragma unroll
         for (int x = 0; x < RB; ++x) {
             const uint32_t r = rr + 4u * (uint32_t)(b + x);
             if (r >= rows_here) continue;
             const float* st = stage_tile + r * 33 + cc;
             const float4 own = make_float4(st[0], st[1], st[2], st[3]);
-            *reinterpret_cast<float4*>(own_blk + (uint64_t)r * own_ld + c0 + cc) = own;
+            *reinterpret_cast<float4*>(k.own_blk + (uint64_t)r * k.own_ld + k.c0 + cc) = own;
+            float4 v[SP];
 #pragma unroll
-            for (int s = 0; s < SP; ++s) if ((uint32_t)s == mine) v[x][s] = own;
+            for (int s = 0; s < SP; ++s) {
+                const float4 lo = o[x][s > 0 ? s - 1 : 0], hi = o[x][s < NO ? s : NO - 1];   // slice s sits in slot s - 1 or s
+                v[s] = (uint32_t)s == k.mine ? own : ((uint32_t)s > k.mine ? lo : hi);
+            }
 #pragma unroll
             for (int w = 1; w < SP; w *= 2)
 #pragma unroll
-                for (int s = 0; s < SP; s += 2 * w) {
-                    v[x][s].x += v[x][s + w].x; v[x][s].y += v[x][s + w].y; v[x][s].z += v[x][s + w].z; v[x][s].w += v[x][s + w].w;
-                }
-            const uint64_t at = c_off + (uint64_t)(row0 + r) * ldc + c0 + cc;
-            if (BF16) *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(c_base) + at) =
-                          make_uint2(pack_bf16(v[x][0].x, v[x][0].y), pack_bf16(v[x][0].z, v[x][0].w));
-            else      *reinterpret_cast<float4*>(static_cast<float*>(c_base) + at) = v[x][0];
+                for (int s = 0; s < SP; s += 2 * w) { v[s].x += v[s + w].x; v[s].y += v[s + w].y; v[s].z += v[s + w].z; v[s].w += v[s + w].w; }
+            const uint64_t at = k.c_off + (uint64_t)(k.row0 + r) * k.ldc + k.c0 + cc;
+            if (BF16) *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(k.c_base) + at) =
+                          make_uint2(pack_bf16(v[0].x, v[0].y), pack_bf16(v[0].z, v[0].w));
+            else      *reinterpret_cast<float4*>(static_cast<float*>(k.c_base) + at) = v[0];
         }
     }
+    __syncwarp();
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kExecThreads, 1)
@@ -539,43 +573,42 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
             for (uint32_t c = 0; c < nchunk; ++c) {
+                const uint32_t q = (c * 32u >= split) ? 1u : 0u;             // (split is a multiple of 32 when a second segment exists)
+                const TileSeg& sg = h.seg[q];
+                const bool live_chunk = rows_here && sg.live && c * 32u < cols;   // warp-uniform
+                const uint32_t ct = c * 32u;                 // chunk's first column in the half-tile ...
+                const uint32_t c0 = ct - (q ? split : 0u);   // ... and in its quadrant
+                if (live_chunk && sum_now[q]) {
+                    // (cells exist only where float4 accesses are aligned and columns come in fours)
+                    SummedChunk k;
+                    k.refs = refs[q]; k.nslices = nslices; k.mine = kslice; k.partials = P.partials;
+                    k.own_blk = P.partials + sg.out_off + (uint64_t)row0 * sg.ld; k.own_ld = sg.ld;
+                    k.row0 = row0; k.rows_here = rows_here; k.c0 = c0; k.cols = width[q];
+                    k.c_base = P.c_ptrs[gemm]; k.c_off = c_off + (q ? split : 0u); k.ldc = ldc;
+                    k.taddr = taddr + ct; k.last_chunk = (c + 1 == nchunk); k.acc_empty_leader = acc_empty_leader;
+                    if (nslices <= 2) { if (out_bf16) summed_chunk<2, true>(k, stage_tile, lane); else summed_chunk<2, false>(k, stage_tile, lane); }
+                    else if (nslices <= 4) { if (out_bf16) summed_chunk<4, true>(k, stage_tile, lane); else summed_chunk<4, false>(k, stage_tile, lane); }
+                    else { if (out_bf16) summed_chunk<8, true>(k, stage_tile, lane); else summed_chunk<8, false>(k, stage_tile, lane); }
+                    continue;
+                }
                 uint32_t v[32];
-                tmem_ld_32x32(taddr + c * 32u, v);
+                tmem_ld_32x32(taddr + ct, v);
                 tmem_ld_wait();
                 if (c + 1 == nchunk) {                       // slot fully read: hand it back to the leader
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
                 }
-                const uint32_t q = (c * 32u >= split) ? 1u : 0u;             // (split is a multiple of 32 when a second segment exists)
-                const TileSeg& sg = h.seg[q];
-                if (rows_here == 0 || !sg.live || c * 32u >= cols) continue; // warp-uniform
+                if (!live_chunk) continue;
 #pragma unroll
                 for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
                 __syncwarp();
-                const uint32_t ct = c * 32u;                 // chunk's first column in the half-tile ...
-                const uint32_t c0 = ct - (q ? split : 0u);   // ... and in its quadrant
                 const uint32_t ld = direct ? ldc : sg.ld;
                 const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg.out_off + (uint64_t)row0 * sg.ld + c0;
                 float* out_f32 = (direct ? static_cast<float*>(P.c_ptrs[gemm]) : P.partials) + out_off;
                 __nv_bfloat16* out_b16 = static_cast<__nv_bfloat16*>(P.c_ptrs[gemm]) + out_off;
                 const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
-                if (sum_now[q]) {
-                    // (cells exist only where float4 accesses are aligned and columns come in fours)
-                    void* cb = P.c_ptrs[gemm];
-                    const uint64_t cq = c_off + (q ? split : 0u);
-                    float* own = P.partials + sg.out_off + (uint64_t)row0 * sg.ld;
-                    if (nslices <= 2) {
-                        if (out_bf16) store_chunk_summed<2, true>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
-                        else          store_chunk_summed<2, false>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
-                    } else if (nslices <= 4) {
-                        if (out_bf16) store_chunk_summed<4, true>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
-                        else          store_chunk_summed<4, false>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
-                    } else {
-                        if (out_bf16) store_chunk_summed<8, true>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
-                        else          store_chunk_summed<8, false>(stage_tile, refs[q], nslices, kslice, P.partials, own, sg.ld, row0, rows_here, c0, width[q], cb, cq, ldc, lane);
-                    }
-                } else if (vec_ok && ct + 32u <= cols) {
+                if (vec_ok && ct + 32u <= cols) {
                     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
 #pragma unroll
                     for (uint32_t r = rr; r < 32u; r += 4u) {

@@ -135,7 +135,9 @@ int repair_memory(const Rect& r, const cleave_device_t& d, const cleave_plan_opt
     return rc ? rc : repair_memory(b, d, o, out);
 }
 
-int plan_one(const cleave_gemm_t& g, const std::vector<cleave_device_t>& devs, const cleave_plan_opts_t& o,
+// level_cells: output cells of all GEMMs of this GEMM's DAG level together (they run in parallel over the
+// same devices, so K is split for fan-out only when the whole level has fewer cells than devices)
+int plan_one(const cleave_gemm_t& g, const std::vector<cleave_device_t>& devs, const cleave_plan_opts_t& o, uint64_t level_cells,
              uint32_t* S_out, uint64_t* tstar_out, std::vector<Rect>& rects) {
     const uint32_t D = (uint32_t)devs.size();
     const uint32_t Mg = (uint32_t)cdiv(g.M, o.gran_m), Ng = (uint32_t)cdiv(g.N, o.gran_n), Kg = (uint32_t)cdiv(g.K, o.gran_k);
@@ -144,7 +146,7 @@ int plan_one(const cleave_gemm_t& g, const std::vector<cleave_device_t>& devs, c
         S = s_limit = std::max(1u, std::min(o.ksplit, Kg));
     } else {
         uint64_t depth = o.kslice_max ? cdiv(g.K, o.kslice_max) : 1;
-        uint64_t fan = cdiv(D, (uint64_t)Mg * Ng);
+        uint64_t fan = cdiv(D, level_cells);
         s_limit = std::min(o.ksplit_cap, Kg);
         S = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(std::max(depth, fan), s_limit));
     }
@@ -285,10 +287,12 @@ int plan_build(cleave_plan_s& p) {
             d.ul_lat_ns > (1ull << 40))
             return CLEAVE_E_INVAL;
     }
+    std::map<uint32_t, uint64_t> level_cells;
+    for (const auto& g : p.gemms) level_cells[g.level] += cdiv(g.M, p.opts.gran_m) * cdiv(g.N, p.opts.gran_n);
     for (uint32_t gi = 0; gi < p.gemms.size(); ++gi) {
         std::vector<Rect> rects;
         uint32_t S = 0; uint64_t tstar = 0;
-        rc = plan_one(p.gemms[gi], p.devices, p.opts, &S, &tstar, rects);
+        rc = plan_one(p.gemms[gi], p.devices, p.opts, level_cells[p.gemms[gi].level], &S, &tstar, rects);
         if (rc) return rc;
         p.ksplit.push_back(S);
         p.tstar.push_back(tstar);

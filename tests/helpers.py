@@ -14,7 +14,7 @@ TASK_FIELDS = ("id", "gemm", "dev", "parent", "m0", "m1", "n0", "n1", "k0", "k1"
 
 
 def oracle_gemms(w):
-    return [Gemm(g.M, g.N, g.K, g.transA, g.transB) for g in w.gemms]
+    return [Gemm(g.M, g.N, g.K, g.transA, g.transB, getattr(g, "level", 0)) for g in w.gemms]
 
 
 def oracle_plan_for(w, **opts):

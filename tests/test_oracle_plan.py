@@ -125,6 +125,13 @@ def test_auto_ksplit():
     assert plan([Gemm(256, 256, 4096)], devs[:4], Opts(kslice_max=2048)).ksplit == [2]
     # more devices than output cells -> split K so that all can work (2x2 cells, 8 devices)
     assert plan([Gemm(256, 256, 512)], devs, Opts()).ksplit == [2]
+    # ... unless the GEMM's level holds enough cells for every device: four such GEMMs in one level are 16
+    # cells for 8 devices (no split), the same four in four levels are split as before
+    four = [Gemm(256, 256, 512, level=0)] * 4
+    assert plan(four, devs, Opts()).ksplit == [1, 1, 1, 1]
+    assert plan([Gemm(256, 256, 512, level=i) for i in range(4)], devs, Opts()).ksplit == [2, 2, 2, 2]
+    assert plan([Gemm(256, 256, 512, level=0), Gemm(256, 256, 512, level=0), Gemm(256, 256, 512, level=1)], devs,
+                Opts()).ksplit == [1, 1, 2]
     # K-slices are consecutive, granule aligned, sizes differ by at most one granule
     p = plan([Gemm(256, 256, 11008)], devs[:4], Opts())
     ranges = sorted({(t.k0, t.k1) for t in p.tasks})

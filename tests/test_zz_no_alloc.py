@@ -31,7 +31,7 @@ def _both_ways(w, **opts):
 def test_two_calls_in_a_row_match_cleave_assemble():
     # first call: several K-slices and slice-count classes; second call: a different, smaller plan
     # whose tables overwrite only the front of the array the first call filled
-    p1, run1 = _both_ways(ci.config(2, 4))
+    p1, run1 = _both_ways(ci.config(2, 4), kslice_max=512)
     assert max(p1.ksplit(i) for i in range(p1.n_gemms)) >= 2
     _both_ways(ci.config(1))
     # and the first plan again, after its tables were overwritten
