@@ -24,7 +24,7 @@ constexpr uint32_t kAccCols = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSchedSlots = 4;
 constexpr int kTileWords16 = sizeof(TileDesc) / 16;   // 16-byte words of a work-list entry
-constexpr uint32_t kEpiStageFloats = 32 * 33;        // per epilogue warp: padded 32 x 32 transpose tile
+constexpr uint32_t kEpiStageFloats = 32 * 32;        // per epilogue warp: 32 x 32 fp32 staging tile (4 KB, 16-byte chunks XOR-swizzled by row)
 
 constexpr int kTmaWarp = 0, kMmaWarp = 1, kSchedWarp = 2, kEpiWarp0 = 4;
 constexpr int kEpiWarpsPerGroup = 4, kEpiWarps = 2 * kEpiWarpsPerGroup;   // group g drains accumulator slot g

@@ -171,6 +171,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// Staging tile of an epilogue warp: 32 rows x 32 fp32, row r at r * 128 bytes, its eight 16-byte chunks
+// stored at chunk position j ^ (r & 7) (the 128-byte swizzle pattern): a lane writing its own row and
+// 8 lanes reading one row both touch all 32 banks once, so neither direction has bank conflicts.
+__device__ __forceinline__ void stage_row(float* stage_tile, uint32_t row, const uint32_t (&v)[32]) {
+    float4* base = reinterpret_cast<float4*>(stage_tile) + row * 8u;
+#pragma unroll
+    for (uint32_t j = 0; j < 8; ++j)
+        base[j ^ (row & 7u)] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+}
+__device__ __forceinline__ float4 staged_f4(const float* stage_tile, uint32_t row, uint32_t col4) {      // columns 4*col4 .. +3
+    return reinterpret_cast<const float4*>(stage_tile)[row * 8u + (col4 ^ (row & 7u))];
+}
+__device__ __forceinline__ float staged_f(const float* stage_tile, uint32_t row, uint32_t col) {
+    return stage_tile[row * 32u + (((col >> 2) ^ (row & 7u)) << 2) + (col & 3u)];
+}
+
 // bytes CTA with `rows` valid rows loads per K-block of a pair whose MMA is n_mma columns wide
 __device__ __forceinline__ uint32_t stage_bytes(uint32_t rows, uint32_t n_mma) {
     const uint32_t nsub_a = (rows + kSubRows - 1) / kSubRows;
@@ -296,8 +312,7 @@ __device__ __forceinline__ void summed_chunk(const SummedChunk& k, float* stage_
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(k.acc_empty_leader);
         }
-#pragma unroll
-        for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
+        stage_row(stage_tile, lane, v);
     }
     __syncwarp();
 #pragma unroll
@@ -307,8 +322,7 @@ __device__ __forceinline__ void summed_chunk(const SummedChunk& k, float* stage_
         for (int x = 0; x < RB; ++x) {
             const uint32_t r = rr + 4u * (uint32_t)(b + x);
             if (r >= rows_here) continue;
-            const float* st = stage_tile + r * 33 + cc;
-            const float4 own = make_float4(st[0], st[1], st[2], st[3]);
+            const float4 own = staged_f4(stage_tile, r, lane & 7u);
             *reinterpret_cast<float4*>(k.own_blk + (uint64_t)r * k.own_ld + k.c0 + cc) = own;
             float4 v[SP];
 #pragma unroll
@@ -411,10 +425,8 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             if (flags & TILE_END) break;
             const CUtensorMap* map_a = P.maps + kMapsPerGemm * gemm;
             const CUtensorMap* map_b = map_a + 1;
-            if (gemm != last_gemm) {
-                for (int x = 0; x < kMapsPerGemm; ++x) tensormap_acquire(map_a + x);
-                last_gemm = gemm;
-            }
+            const bool new_gemm = gemm != last_gemm;     // (each issuing lane acquires the one map it uses, below)
+            last_gemm = gemm;
             if (level != last_level) {
                 // operands of this level may have been written by other SMs a moment ago (ordinary stores, seen
                 // through the scheduler's acquire): order them before this thread's asynchronous loads
@@ -441,6 +453,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             const bool my_mn = is_a ? (flags & TILE_A_MN) : (flags & TILE_B_MN);
             const int32_t my_x = (int32_t)((is_a ? a_x : b_x) + j * kSubRows);
             const uint32_t my_off = (is_a ? 0u : kPairABytes) + j * kSubBytes;
+            if (new_gemm && (is_a || is_b)) tensormap_acquire(my_map);
             for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const uint32_t s = it % kPairStages, ph = (it / kPairStages) & 1u;
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait_cl(smem_u32(&sh.empty[s]), ph ^ 1u, W))) { ok = false; break; }
@@ -600,8 +613,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
                 }
                 if (!live_chunk) continue;
-#pragma unroll
-                for (int x = 0; x < 32; ++x) stage_tile[lane * 33 + x] = __uint_as_float(v[x]);
+                stage_row(stage_tile, lane, v);
                 __syncwarp();
                 const uint32_t ld = direct ? ldc : sg.ld;
                 const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg.out_off + (uint64_t)row0 * sg.ld + c0;
@@ -613,17 +625,16 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
 #pragma unroll
                     for (uint32_t r = rr; r < 32u; r += 4u) {
                         if (r < rows_here) {
-                            const float* src = stage_tile + r * 33 + cc;
+                            const float4 x = staged_f4(stage_tile, r, lane & 7u);
                             if (to_bf16) *reinterpret_cast<uint2*>(out_b16 + (uint64_t)r * ld + cc) =
-                                             make_uint2(pack_bf16(src[0], src[1]), pack_bf16(src[2], src[3]));
-                            else         *reinterpret_cast<float4*>(out_f32 + (uint64_t)r * ld + cc) =
-                                             make_float4(src[0], src[1], src[2], src[3]);
+                                             make_uint2(pack_bf16(x.x, x.y), pack_bf16(x.z, x.w));
+                            else         *reinterpret_cast<float4*>(out_f32 + (uint64_t)r * ld + cc) = x;
                         }
                     }
                 } else if (ct + lane < cols) {
 #pragma unroll 8
                     for (uint32_t r = 0; r < rows_here; ++r) {
-                        const float x = stage_tile[r * 33 + lane];
+                        const float x = staged_f(stage_tile, r, lane);
                         if (to_bf16) out_b16[(uint64_t)r * ld + lane] = __float2bfloat16_rn(x);
                         else         out_f32[(uint64_t)r * ld + lane] = x;
                     }

@@ -169,11 +169,10 @@ cudaError_t launch_verify(const cleave_task_t* tasks, uint32_t n_tasks, const cl
                           const void* const* ab_ptrs, const float* partials, float* const* c_ptrs, int fused, uint64_t seed,
                           float tol, float4* out, unsigned int* n_bad, uint32_t sign_bytes, cudaStream_t st) {
     if (!n_tasks) return cudaSuccess;
-    static uint32_t configured = 0;
-    if (sign_bytes > 40 * 1024 && sign_bytes > configured) {
+    if (sign_bytes > 40 * 1024) {
+        // the attribute belongs to the current device's copy of the kernel: set it on every such launch
         cudaError_t e = cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sign_bytes);
         if (e != cudaSuccess) return e;
-        configured = sign_bytes;
     }
     verify_kernel<<<n_tasks, kVerifyThreads, sign_bytes, st>>>(tasks, n_tasks, gemms, ksplit, ab_ptrs, partials, c_ptrs, fused,
                                                                (unsigned long long)seed, tol, out, n_bad);

@@ -43,6 +43,47 @@ def test_two_calls_in_a_row_match_cleave_assemble():
         assert np.array_equal(a.view(np.uint32), b.cpu().numpy().view(np.uint32))
 
 
+def test_no_device_memory_is_taken_by_the_call():
+    """The property in the entry point's name: a plan that has never touched the device is assembled
+    through the fixed array, and neither the driver's free-memory figure nor torch's allocator moves."""
+    import torch
+    import paper_2512_22142_b200 as cl
+    w = ci.config(2, 4)
+    ts = ci.make_tensors(w)
+    p = lib_plan_for(w, kslice_max=512)
+    run = GpuRun(w, ts, p)
+    run.exec(); run.assemble(); p.check_status()
+    ref = run.results()
+    warm = lib_plan_for(ci.config(1))                       # first use of the array on this device, if it is the first
+    x = torch.zeros(warm.arena_elems, dtype=torch.float32, device="cuda:0")
+    warm.assemble_static(x, [torch.zeros(256, 768, dtype=torch.float32, device="cuda:0")])
+    fresh = lib_plan_for(w, kslice_max=512)                 # same plan, host tables only: no device state yet
+    out = [torch.full_like(c, float("nan")) for c in run.C]
+    torch.cuda.synchronize()
+    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    fresh.assemble_static(run.partials, out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    for g, a, b in zip(w.gemms, ref, out):
+        assert np.array_equal(a.view(np.uint32), b.cpu().numpy().view(np.uint32)), g.name
+    # two calls back to back on one stream, nothing in between: the second call's tables wait for the first's kernels
+    out2 = [torch.full_like(c, float("nan")) for c in run.C]
+    fresh.assemble_static(run.partials, out)
+    fresh.assemble_static(run.partials, out2)
+    torch.cuda.synchronize()
+    for a, b in zip(ref, out2):
+        assert np.array_equal(a.view(np.uint32), b.cpu().numpy().view(np.uint32))
+    # after a fused execution part of the result sits in the C that execution was given: another C is refused
+    run.exec_fused()
+    with pytest.raises(cl.CleaveError) as e:
+        p.assemble_static(run.partials, out)
+    assert e.value.code == -1
+    p.assemble_static(run.partials, run.C)
+    for a, b in zip(ref, run.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
 def test_oversized_plan_is_refused_before_any_launch():
     import paper_2512_22142_b200 as cl
     p = lib_plan_for(ci.config(3))                   # ~3 MiB of tables: beyond the fixed array
