@@ -96,6 +96,12 @@ typedef struct {
     uint32_t ksplit_cap;              /* upper limit of the automatic choice (default 8)          */
     uint32_t reissue_fanout;          /* pieces a failed task is cut into (default 4)             */
     uint32_t b_in, b_out;             /* bytes per input / partial-output element (2, 4)          */
+    /* Tail-aware cost (Appendix C, "Tail-Aware Cost Model"): with tail_alpha_milli > 1000 every
+     * latency overhead L^d_k, L^u_k is taken as the scale of a Pareto distribution with shape
+     * alpha = tail_alpha_milli / 1000 and enters the cost model with its conditional value-at-risk
+     * over the worst beta = tail_beta_ppm / 10^6 of outcomes (Eq. 24):
+     * L * alpha / ((alpha - 1) * beta^(1/alpha)), rounded up to whole ns.  0 = off (default). */
+    uint32_t tail_alpha_milli, tail_beta_ppm;
 } cleave_plan_opts_t;
 
 typedef struct cleave_plan_s cleave_plan_t;   /* opaque; owned by the library until cleave_destroy */

@@ -66,3 +66,25 @@ def lower_bound_ns(gemm_flops: int, devices) -> int:
     single GEMM.  Returned: floor(W / sum F) in ns (a lower bound on any plan's makespan)."""
     total_f = sum(d.flops_mflops for d in devices)
     return (gemm_flops * 1000) // total_f
+
+
+def tail_latency_scale_q20(alpha_milli: int, beta_ppm: int) -> int:
+    """Tail-aware latency (Appendix C, Eqs. 20, 23, 24): a latency overhead is modelled as Pareto
+    with shape alpha and scale x_m = the device's stated overhead, and enters the cost with its
+    conditional value-at-risk over the worst beta-fraction of outcomes,
+        CVaR_beta[L] = x_m / beta^(1/alpha) * alpha / (alpha - 1)          (alpha > 1).
+    Returned: floor(2^20 * CVaR_beta[L] / x_m), from alpha in thousandths and beta in millionths.
+    (One floating-point power; the integer result is what plans are built from.)"""
+    if alpha_milli <= 1000 or not (0 < beta_ppm <= 1_000_000):
+        raise ValueError("tail model needs alpha > 1 and 0 < beta <= 1")
+    import math
+    a = alpha_milli / 1000.0
+    b = beta_ppm / 1000000.0
+    f = (a / (a - 1.0)) * math.pow(b, -1.0 / a)
+    return int(math.floor(f * 1048576.0))
+
+
+def tail_aware(dev: Device, alpha_milli: int, beta_ppm: int) -> Device:
+    """The device with both latency overheads replaced by their CVaR (rounded up to whole ns)."""
+    q = tail_latency_scale_q20(alpha_milli, beta_ppm)
+    return dev._replace(dl_lat_ns=ceil_div(dev.dl_lat_ns * q, 1 << 20), ul_lat_ns=ceil_div(dev.ul_lat_ns * q, 1 << 20))

@@ -26,7 +26,7 @@ from dataclasses import dataclass, field, replace
 from math import isqrt
 from typing import List, Optional, Sequence
 
-from .cost import Device, ceil_div, task_cost, task_mem, NS
+from .cost import Device, ceil_div, tail_aware, task_cost, task_mem, NS
 
 T_MAX = 1 << 50
 
@@ -65,6 +65,8 @@ class Opts:
     reissue_fanout: int = 4
     b_in: int = 2
     b_out: int = 4
+    tail_alpha_milli: int = 0      # > 1000: tail-aware latencies (Appendix C), Pareto shape in thousandths; 0 = off
+    tail_beta_ppm: int = 50_000     # worst fraction of outcomes the CVaR averages over, in millionths (0.05)
 
 
 @dataclass
@@ -307,6 +309,9 @@ def plan(gemms: Sequence[Gemm], devices: Sequence[Device], opts: Opts = Opts()) 
     """Every GEMM is planned independently over the same device list (each GEMM is its own
     dispatch round; a schedule is computed when the device set changes and kept until it changes
     again, Section 3.2)."""
+    if opts.tail_alpha_milli:
+        # tail-aware cost (Appendix C, Eq. 23): every latency overhead enters with its CVaR (Eq. 24)
+        devices = [tail_aware(d, opts.tail_alpha_milli, opts.tail_beta_ppm) for d in devices]
     p = Plan(list(gemms), list(devices), opts)
     per_gemm = []
     cells = {}

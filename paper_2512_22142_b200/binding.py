@@ -29,7 +29,7 @@ assert DEVICE_DTYPE.itemsize == 48 and GEMM_DTYPE.itemsize == 24 and TASK_DTYPE.
 
 class Opts(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("gran_m", "gran_n", "gran_k", "kslice_max", "ksplit",
-                                          "ksplit_cap", "reissue_fanout", "b_in", "b_out")]
+                                          "ksplit_cap", "reissue_fanout", "b_in", "b_out", "tail_alpha_milli", "tail_beta_ppm")]
 
 
 _vp, _u32, _u64, _i = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int

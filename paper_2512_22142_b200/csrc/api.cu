@@ -319,6 +319,8 @@ void cleave_plan_opts_default(cleave_plan_opts_t* o) {
     o->reissue_fanout = 4;
     o->b_in = 2;
     o->b_out = 4;
+    o->tail_alpha_milli = 0;
+    o->tail_beta_ppm = 50000;
 }
 
 static int new_plan(const cleave_gemm_t* g, uint32_t n_gemms, const cleave_plan_opts_t* o, cleave_plan_s** out) {

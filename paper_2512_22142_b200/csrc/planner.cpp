@@ -11,6 +11,7 @@
 //   K-slices; split whatever still violates the memory constraint.
 #include <algorithm>
 #include <array>
+#include <cmath>
 #include <cstring>
 #include <map>
 #include <numeric>
@@ -281,6 +282,19 @@ int plan_build(cleave_plan_s& p) {
     int rc = validate_common(p);
     if (rc) return rc;
     if (p.devices.empty()) return CLEAVE_E_NO_DEVICES;
+    if (p.opts.tail_alpha_milli) {
+        // tail-aware cost (Appendix C): every latency overhead enters with its conditional value-at-risk
+        // L * alpha / ((alpha - 1) * beta^(1/alpha)); the factor is fixed to 20 fractional bits, the rest is integer
+        if (p.opts.tail_alpha_milli <= 1000 || !p.opts.tail_beta_ppm || p.opts.tail_beta_ppm > 1000000) return CLEAVE_E_INVAL;
+        const double a = p.opts.tail_alpha_milli / 1000.0, b = p.opts.tail_beta_ppm / 1000000.0;
+        const double f = (a / (a - 1.0)) * std::pow(b, -1.0 / a);
+        const uint64_t q = (uint64_t)std::floor(f * 1048576.0);
+        for (auto& d : p.devices) {
+            if (d.dl_lat_ns > (1ull << 40) || d.ul_lat_ns > (1ull << 40)) return CLEAVE_E_INVAL;
+            d.dl_lat_ns = (uint64_t)(((u128)d.dl_lat_ns * q + (1u << 20) - 1) >> 20);
+            d.ul_lat_ns = (uint64_t)(((u128)d.ul_lat_ns * q + (1u << 20) - 1) >> 20);
+        }
+    }
     for (const auto& d : p.devices) {
         if (d.mem_bytes > (1ull << 48) || !d.flops_mflops || d.flops_mflops > (1ull << 40) || !d.dl_Bps ||
             d.dl_Bps > (1ull << 40) || !d.ul_Bps || d.ul_Bps > (1ull << 40) || d.dl_lat_ns > (1ull << 40) ||

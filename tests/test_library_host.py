@@ -45,6 +45,29 @@ def test_planner_equals_oracle(cl, cfg, scale):
         assert p.tstar_ns(gi) == op.t_star[gi]
 
 
+@pytest.mark.parametrize("alpha_milli,beta_ppm", [(3000, 50_000), (1500, 10_000), (2500, 200_000)])
+def test_tail_aware_planner_equals_oracle(cl, alpha_milli, beta_ppm):
+    """Appendix C's tail-aware cost (latencies at their CVaR): same task lists, and levels of a DAG
+    cost what the oracle's level recursion says."""
+    from oracle.levels import plan_level_costs
+    w = ci.config(3, 4)
+    kw = dict(tail_alpha_milli=alpha_milli, tail_beta_ppm=beta_ppm)
+    p, op = lib_plan_for(w, **kw), oracle_plan_for(w, **kw)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    base = lib_plan_for(w)
+    assert all(p.tstar_ns(i) == op.t_star[i] and p.tstar_ns(i) > base.tstar_ns(i) for i in range(p.n_gemms))
+    gemms, tensors, produced = ci.two_branch_chain(512, 256, 384, 256)
+    wc = ci.Workload("chain", gemms, tensors, n_devices=9, mem_range=(64 * ci.MB, ci.GB), produced=produced)
+    pc, oc = lib_plan_for(wc, **kw), oracle_plan_for(wc, **kw)
+    assert np.array_equal(task_matrix_lib(pc), task_matrix_oracle(oc))
+    want = plan_level_costs(oc, [g.level for g in gemms])
+    assert pc.num_levels == 3 and pc.step_makespan_ns == want[-1]
+    assert [pc.level_makespan_ns(s) for s in range(3)] == [want[0], want[1] - want[0], want[2] - want[1]]
+    with pytest.raises(cl.CleaveError) as e:
+        lib_plan_for(w, tail_alpha_milli=1000)              # infinite mean: no CVaR
+    assert e.value.code == -1
+
+
 @pytest.mark.parametrize("seed", range(10))
 def test_planner_equals_oracle_random_small(cl, seed):
     rng = np.random.default_rng(100 + seed)
@@ -126,5 +149,5 @@ def test_header_is_plain_c_and_defaults_agree_with_oracle(cl, tmp_path):
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
     assert subprocess.run([str(exe)]).returncode == 0
     o, ref = cl.default_opts(), Opts()
-    for name in ("gran_m", "gran_n", "gran_k", "kslice_max", "ksplit", "ksplit_cap", "reissue_fanout", "b_in", "b_out"):
+    for name in ("gran_m", "gran_n", "gran_k", "kslice_max", "ksplit", "ksplit_cap", "reissue_fanout", "b_in", "b_out", "tail_alpha_milli", "tail_beta_ppm"):
         assert getattr(o, name) == getattr(ref, name), name
