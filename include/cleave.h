@@ -36,7 +36,7 @@ extern "C" {
 /* ---- error codes ------------------------------------------------------------------------- */
 #define CLEAVE_OK              0
 #define CLEAVE_E_INVAL        -1   /* bad argument (null pointer, zero size, value out of range)   */
-#define CLEAVE_E_UNSUPPORTED  -2   /* valid plan the kernels cannot run (alignment, slice count)   */
+#define CLEAVE_E_UNSUPPORTED  -2   /* valid plan or option the kernels cannot run (see the calls)  */
 #define CLEAVE_E_INFEASIBLE   -3   /* no plan satisfies the memory constraint                      */
 #define CLEAVE_E_NO_DEVICES   -4   /* empty device list, or no surviving device for a GEMM         */
 #define CLEAVE_E_RANGE        -5   /* task id >= number of tasks                                   */
@@ -161,8 +161,13 @@ CLEAVE_API int cleave_set_drops(cleave_plan_t* p, const uint32_t* ids, uint32_t 
  * A'_{s,p,k} o B'_{s,p,k}, a block of O_s).  Marks each finished task in the plan's bookkeeping.
  *   A, B [host arrays of n_gemms device pointers]; partials [device, >= arena_elems floats,
  *   128-byte aligned].  The first call on a plan creates its device mirrors (allocates).
- * Requirements on the plan (else E_UNSUPPORTED): k0 a multiple of 64 and k1 a multiple of 64 or
- * equal to K; m0 a multiple of 8 when transA = 1; n0 a multiple of 8 when transB = 0.
+ * The tensor-core kernel needs: k0 a multiple of 64 and k1 a multiple of 64 or equal to K; m0 a
+ * multiple of 8 when transA = 1; n0 a multiple of 8 when transB = 0; lda, ldb multiples of 8.  A
+ * plan with a task off these rules (hand-picked granules, ragged uniform grids; the default
+ * granules never produce one) is run by a plain CUDA-core kernel instead: same blocks, bookkeeping
+ * and churn path, much slower, every block to the arena (the fused calls below then behave as
+ * cleave_exec and leave C to cleave_assemble); such a plan must have a single DAG level
+ * (else E_UNSUPPORTED).
  * Errors: E_INVAL, E_UNSUPPORTED, E_CUDA, E_NOMEM. */
 CLEAVE_API int cleave_exec(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
                 void* stream);

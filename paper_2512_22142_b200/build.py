@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB_DIR = os.path.join(PKG, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libcleave.so")
-SOURCES = ["planner.cpp", "kernels.cu", "kernels_pair.cu", "kernels_verify.cu", "api.cu"]
+SOURCES = ["planner.cpp", "kernels.cu", "kernels_pair.cu", "kernels_verify.cu", "kernels_simple.cu", "api.cu"]
 HEADERS = ["plan_internal.hpp", "kernels.cuh", "ptx.cuh", os.path.join(ROOT, "include", "cleave.h")]
 
 

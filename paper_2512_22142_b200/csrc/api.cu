@@ -222,7 +222,8 @@ int update_maps(cleave_plan_s* p, const void* const* A, const void* const* B, cu
 int check_exec_args(cleave_plan_s* p, const void* const* A, const void* const* B, float* partials) {
     if (!p || !A || !B || !partials) return CLEAVE_E_INVAL;
     if ((uintptr_t)partials & 127) return CLEAVE_E_INVAL;
-    if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
+    // plans off the tensor-core kernel's alignment rules run on the plain kernel, one DAG level only
+    if (p->exec_unsupported && p->n_levels > 1) return CLEAVE_E_UNSUPPORTED;
     for (const auto& g : p->gemms) {
         const uint32_t need_a = g.transA ? g.M : g.K, need_b = g.transB ? g.K : g.N;
         if (g.lda < need_a || g.ldb < need_b) return CLEAVE_E_INVAL;
@@ -267,6 +268,41 @@ int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, bool fre
         CU_TRY(cudaEventRecord(d->ev[1], st));
         d->ev_exec = true;
     }
+    return 0;
+}
+
+// Device copies of the GEMM records and of the operand pointers (block verification and the plain exec kernel).
+int upload_gemm_tables(cleave_plan_s* p, const void* const* A, const void* const* B, cudaStream_t st) {
+    DeviceState* d = p->dev;
+    const size_t n = p->gemms.size();
+    if (!d->gemm_table) {
+        RC_TRY(dev_alloc(&d->gemm_table, n)); RC_TRY(dev_alloc(&d->ksplit_table, n)); RC_TRY(dev_alloc(&d->ab_ptrs, 2 * n));
+        CU_TRY(cudaMemcpyAsync(d->gemm_table, p->gemms.data(), n * sizeof(cleave_gemm_t), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->ksplit_table, p->ksplit.data(), n * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    }
+    std::vector<const void*> ab(2 * n);
+    for (size_t i = 0; i < n; ++i) {
+        if (!A[i] || !B[i] || ((uintptr_t)A[i] & 15) || ((uintptr_t)B[i] & 15)) return CLEAVE_E_INVAL;
+        ab[2 * i] = A[i]; ab[2 * i + 1] = B[i];
+    }
+    CU_TRY(cudaMemcpyAsync(d->ab_ptrs, ab.data(), ab.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
+    return 0;
+}
+
+// The plain kernel over tasks [task_begin, end): every block goes to the arena (cleave_assemble finishes C).
+int run_tasks_plain(cleave_plan_s* p, uint32_t task_begin, bool fresh, const void* const* A, const void* const* B,
+                    float* partials, cudaStream_t st) {
+    DeviceState* d = p->dev;
+    RC_TRY(upload_gemm_tables(p, A, B, st));
+    if (fresh) {
+        CU_TRY(cudaMemsetAsync(d->words + 1, 0, sizeof(unsigned int), st));          // forget earlier verdicts
+        CU_TRY(cudaMemsetAsync(d->done, 0, d->tasks_n * sizeof(uint32_t), st));
+    }
+    CU_TRY(cudaEventRecord(d->ev[0], st));
+    CU_TRY(launch_exec_simple(d->tasks, task_begin, d->tasks_n, d->gemm_table, d->ab_ptrs, d->dropped, d->ntiles, partials,
+                              p->arena_elems, d->done, d->words + 1, st));
+    CU_TRY(cudaEventRecord(d->ev[1], st));
+    d->ev_exec = true;
     return 0;
 }
 
@@ -405,6 +441,15 @@ int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* 
     if ((flags & (CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH)) && !C) return CLEAVE_E_INVAL;
     if (level_begin > level_end) return CLEAVE_E_INVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (p->exec_unsupported) {
+        // every block to the arena with the plain kernel; C is written by the cleave_assemble that follows
+        if (level_begin != 0 || level_end < p->n_levels) return CLEAVE_E_UNSUPPORTED;
+        try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+        p->mode = (flags & CLEAVE_EXEC_BF16) ? MODE_BF16 : 0u;
+        p->fused = p->finished = false;
+        p->out_bf16 = (p->mode & MODE_BF16) != 0;
+        try { return run_tasks_plain(p, 0, true, A, B, partials, st); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
+    }
     try {
         RC_TRY(sync_device_state(p, st));
         RC_TRY(update_maps(p, A, B, st));
@@ -488,8 +533,16 @@ int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t n, const v
         }
         const uint32_t tiles_before = (uint32_t)p->tiles.size();
         uint32_t first_new = 0;
+        const bool was_plain = p->exec_unsupported != 0;
         RC_TRY(plan_reissue(*p, failed, n, &first_new));
-        if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
+        if (p->exec_unsupported) {
+            // (a plan that ran on the tensor-core kernel and only now gets a piece off its rules is refused: part
+            // of its result may sit in C already)
+            if (p->n_levels > 1 || !was_plain) return CLEAVE_E_UNSUPPORTED;
+            p->fused = p->finished = false;
+            RC_TRY(sync_device_state(p, st));
+            return run_tasks_plain(p, first_new, false, A, B, partials, st);
+        }
         RC_TRY(sync_device_state(p, st));
         RC_TRY(update_maps(p, A, B, st));
         p->finished = false;                           // cells that lost a block are summed by cleave_assemble
@@ -514,17 +567,12 @@ int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, 
                   float tol, uint32_t* n_bad, void* stream) {
     if (!p || !A || !B || !partials || !n_bad || !(tol >= 0.f)) return CLEAVE_E_INVAL;
     for (const auto& g : p->gemms) if ((g.K % 4) || (g.lda % 8) || (g.ldb % 8)) return CLEAVE_E_UNSUPPORTED;
-    if (p->exec_unsupported) return CLEAVE_E_UNSUPPORTED;
     if (p->fused && p->out_bf16) return CLEAVE_E_UNSUPPORTED;      // blocks written to C as bf16 are not checked
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     DeviceState* d = p->dev;
     const size_t n = p->gemms.size();
-    if (!d->gemm_table) {
-        RC_TRY(dev_alloc(&d->gemm_table, n)); RC_TRY(dev_alloc(&d->ksplit_table, n)); RC_TRY(dev_alloc(&d->ab_ptrs, 2 * n));
-        CU_TRY(cudaMemcpyAsync(d->gemm_table, p->gemms.data(), n * sizeof(cleave_gemm_t), cudaMemcpyHostToDevice, st));
-        CU_TRY(cudaMemcpyAsync(d->ksplit_table, p->ksplit.data(), n * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
-    }
+    RC_TRY(upload_gemm_tables(p, A, B, st));
     if (d->verify_cap < d->tasks_cap) {
         CU_TRY(cudaStreamSynchronize(st));
         cudaFree(d->verify_out);
@@ -532,16 +580,10 @@ int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, 
         RC_TRY(dev_alloc(&d->verify_out, d->tasks_cap));
         d->verify_cap = d->tasks_cap;
     }
-    std::vector<const void*> ab(2 * n);
     uint32_t sign_bytes = 0;
-    for (size_t i = 0; i < n; ++i) {
-        if (!A[i] || !B[i] || ((uintptr_t)A[i] & 15) || ((uintptr_t)B[i] & 15)) return CLEAVE_E_INVAL;
-        ab[2 * i] = A[i]; ab[2 * i + 1] = B[i];
-    }
     for (const auto& t : p->tasks) sign_bytes = std::max(sign_bytes, (t.m1 - t.m0) + (t.n1 - t.n0));
     sign_bytes = (sign_bytes + 15) / 16 * 16;
     if (sign_bytes > 200 * 1024) return CLEAVE_E_UNSUPPORTED;
-    CU_TRY(cudaMemcpyAsync(d->ab_ptrs, ab.data(), ab.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
     CU_TRY(cudaMemsetAsync(d->words + 3, 0, sizeof(unsigned int), st));
     CU_TRY(launch_verify(d->tasks, d->tasks_n, d->gemm_table, d->ksplit_table, d->ab_ptrs, partials, reinterpret_cast<float* const*>(d->c_ptrs), p->fused ? 1 : 0,
                          seed, tol, d->verify_out, d->words + 3, sign_bytes, st));

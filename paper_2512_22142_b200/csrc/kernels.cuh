@@ -77,6 +77,10 @@ cudaError_t launch_collect_failed(const cleave_task_t* tasks, const uint32_t* do
 cudaError_t launch_verify(const cleave_task_t* tasks, uint32_t n_tasks, const cleave_gemm_t* gemms, const uint32_t* ksplit,
                           const void* const* ab_ptrs, const float* partials, float* const* c_ptrs, int fused, uint64_t seed,
                           float tol, float4* out, unsigned int* n_bad, uint32_t sign_bytes, cudaStream_t st);
+// the sub-GEMMs of tasks [task_begin, task_end) without tensor cores (plans the exec kernel cannot take)
+cudaError_t launch_exec_simple(const cleave_task_t* tasks, uint32_t task_begin, uint32_t task_end, const cleave_gemm_t* gemms,
+                               const void* const* ab_ptrs, const uint8_t* dropped, const uint32_t* ntiles, float* partials,
+                               uint64_t arena_elems, uint32_t* done, unsigned int* status, cudaStream_t st);
 // sp = padded slice count of the vectorised kernel (1, 2, 4, 8, 16, 32), 0 = scalar kernel; out_bf16: C holds bf16
 cudaError_t launch_assemble(const AsmItem* items, const AsmRef* refs, uint32_t item0, uint32_t n_items, uint32_t sp,
                             const float* partials, void* const* Cptr, const uint32_t* ldcs, int out_bf16, cudaStream_t st);

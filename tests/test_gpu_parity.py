@@ -295,14 +295,45 @@ def test_every_task_dropped():
     assert all(np.isfinite(c).all() for c in run.results())
 
 
-def test_unsupported_alignment_is_rejected():
+def test_plans_off_the_alignment_rules_run_on_the_plain_kernel():
+    """K-ranges that do not start on multiples of 64, leading dimensions that are no multiples of 8,
+    blocks that start on odd rows and columns: the tensor-core kernel cannot take such plans, the plain
+    kernel runs them -- same blocks, same bookkeeping, same churn path -- in all three layouts."""
     import torch
-    import paper_2512_22142_b200 as cl
-    gemms, tensors = ci.projection_gemms(64, [("p", 200, 64)], ("fwd",))     # K = 200 in 2 slices of 100
-    p = cl.plan_uniform(gemms, 1, 1, 2)
-    x = torch.zeros(64, 200, dtype=torch.bfloat16, device="cuda:0")
-    wt = torch.zeros(200, 64, dtype=torch.bfloat16, device="cuda:0")
-    part = torch.zeros(p.arena_elems, dtype=torch.float32, device="cuda:0")
-    with pytest.raises(cl.CleaveError) as e:
-        p.exec([x], [wt], part)
-    assert e.value.code == -2
+    gemms, tensors = ci.projection_gemms(90, [("p", 200, 84)])              # K = 200 in 2 slices of 100; N = 84; M = 90
+    w = ci.Workload("off-rules", gemms, tensors, uniform=(3, 2, 2))
+    ts = ci.make_tensors(w, integer=True)
+    p, op = lib_plan_for(w), oracle_plan_for(w)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    A, B = oracle_operands(w, ts)
+    ref = nm.assemble(op, nm.execute(op, A, B))
+    run = GpuRun(w, ts, p)
+    run.exec_fused(); run.assemble(); p.check_status()                      # a fused call falls back to two steps
+    for g, got, want in zip(w.gemms, run.results(), ref):
+        assert np.array_equal(got.astype(np.float64), want), g.name
+    done = p.done_counts()
+    assert all(done[i] == p.task_num_tiles(i) for i in range(p.num_tasks))
+    # churn on the same path
+    failed = np.array([1, 7, 20], dtype=np.uint32)
+    p.set_drops(failed)
+    run.partials.fill_(float("nan"))
+    for c in run.C:
+        c.fill_(float("nan"))
+    run.exec(); run.assemble()
+    assert p.status() == -9 and (p.done_counts()[failed] == 0).all()
+    run.reissue(None)
+    oracle_reissue(op, failed)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    run.assemble()
+    assert p.status() == 0
+    for g, got, want in zip(w.gemms, run.results(), ref):
+        assert np.array_equal(got.astype(np.float64), want), g.name
+    # Gaussian inputs within the path's tolerance
+    ts = ci.make_tensors(w)
+    A, B = oracle_operands(w, ts)
+    p2, op2 = lib_plan_for(w), oracle_plan_for(w)
+    ref = nm.assemble(op2, nm.execute(op2, A, B))
+    run2 = GpuRun(w, ts, p2)
+    run2.exec(); run2.assemble(); p2.check_status()
+    for gi, (g, got, want) in enumerate(zip(w.gemms, run2.results(), ref)):
+        assert_within_tolerance(got, want, nm.abs_bound(A[gi], B[gi]), what=g.name)
