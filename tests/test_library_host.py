@@ -151,3 +151,39 @@ def test_header_is_plain_c_and_defaults_agree_with_oracle(cl, tmp_path):
     o, ref = cl.default_opts(), Opts()
     for name in ("gran_m", "gran_n", "gran_k", "kslice_max", "ksplit", "ksplit_cap", "reissue_fanout", "b_in", "b_out", "tail_alpha_milli", "tail_beta_ppm"):
         assert getattr(o, name) == getattr(ref, name), name
+
+
+def test_levels_and_new_options_on_the_host(cl):
+    """DAG levels, the finishable flag and argument checks that need no device."""
+    from oracle.levels import plan_level_costs
+    gemms, tensors, produced = ci.two_branch_chain(512, 256, 384, 256)
+    w = ci.Workload("chain", gemms, tensors, n_devices=7, mem_range=(64 * ci.MB, ci.GB), produced=produced)
+    p, op = lib_plan_for(w, kslice_max=256), oracle_plan_for(w, kslice_max=256)
+    assert np.array_equal(task_matrix_lib(p), task_matrix_oracle(op))
+    assert p.num_levels == 3
+    want = plan_level_costs(op, [g.level for g in gemms])
+    assert p.step_makespan_ns == want[-1] and p.level_makespan_ns(0) == want[0] and p.level_makespan_ns(7) == 0
+    # on the 128-grid every K-split GEMM can be summed by the exec kernel; one-slice GEMMs have nothing to sum
+    for i in range(p.n_gemms):
+        assert p.finishable(i) == (p.ksplit(i) >= 2)
+    assert not p.finishable(99)
+    # more than 8 K-slices, or N not a multiple of 4, are left to the assembly kernel
+    g1, t1 = ci.projection_gemms(256, [("p", 2048, 256)], ("fwd",))
+    many = cl.plan(g1, ci.make_devices(4, 64 * ci.MB, ci.GB, 0), cl.default_opts(ksplit=12, kslice_max=0, ksplit_cap=32))
+    assert many.ksplit(0) == 12 and not many.finishable(0)
+    # levels beyond the limit are refused when the plan is made
+    class G:
+        def __init__(self, g, level):
+            self.__dict__.update(M=g.M, N=g.N, K=g.K, transA=g.transA, transB=g.transB, lda=g.lda, ldb=g.ldb, level=level)
+    with pytest.raises(cl.CleaveError) as e:
+        cl.plan([G(g1[0], 4096)], ci.make_devices(4, 64 * ci.MB, ci.GB, 0))
+    assert e.value.code == -1
+    ok = cl.plan([G(g1[0], 4095)], ci.make_devices(4, 64 * ci.MB, ci.GB, 0))
+    assert ok.num_levels == 4096
+    # tile counts: a plan on the 128-grid is cut into full 256 x 256 pairs per K-range, whatever its blocks
+    w3 = ci.config(3, 4)
+    p3 = lib_plan_for(w3)
+    pairs = sum(-(-g.M // 256) * -(-g.N // 256) * p3.ksplit(i) for i, g in enumerate(w3.gemms))
+    assert p3.num_tiles == pairs
+    quadrants = sum(p3.task_num_tiles(i) for i in range(p3.num_tasks))
+    assert quadrants == sum(-(-g.M // 128) * -(-g.N // 128) * p3.ksplit(i) for i, g in enumerate(w3.gemms))
