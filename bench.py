@@ -250,7 +250,7 @@ def plan_summary(plan, n_gemms, n_devices):
             "modelled_step_makespan_ms": plan.step_makespan_ns / 1e6}
 
 
-def quick_leg(cl, ci, torch, dev, name, cfg, scale, opts, mode, min_s=0.6, tensors=None, bf16_out=False):
+def quick_leg(cl, ci, torch, dev, name, cfg, scale, opts, mode, min_s=0.6, tensors=None, bf16_out=False, consume=True):
     """Plans the workload, runs it for at least `min_s` seconds untimed, then times the same number of
     steps again: step / exec / assembly times from CUDA events on the launching stream."""
     w = ci.config(cfg, scale)
@@ -268,7 +268,7 @@ def quick_leg(cl, ci, torch, dev, name, cfg, scale, opts, mode, min_s=0.6, tenso
         if mode == "two-step":
             plan.exec_opts(A, B, partials, C, bf16=bf16_out)
         else:
-            plan.exec_opts(A, B, partials, C, direct=True, finish=True, bf16=bf16_out)
+            plan.exec_opts(A, B, partials, C, direct=True, finish=True, bf16=bf16_out, consume=consume)
         plan.assemble(partials, C)
 
     n, t0 = 0, time.perf_counter()
@@ -286,7 +286,7 @@ def quick_leg(cl, ci, torch, dev, name, cfg, scale, opts, mode, min_s=0.6, tenso
         if mode == "two-step":
             plan.exec_opts(A, B, partials, C, bf16=bf16_out)
         else:
-            plan.exec_opts(A, B, partials, C, direct=True, finish=True, bf16=bf16_out)
+            plan.exec_opts(A, B, partials, C, direct=True, finish=True, bf16=bf16_out, consume=consume)
         e[1].record()
         plan.assemble(partials, C)
         e[2].record()
@@ -376,7 +376,8 @@ def run_ours(args):
         if args.two_step:
             plan.exec_opts(A, B, partials, C, bf16=args.bf16_out)
         else:
-            plan.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish, bf16=args.bf16_out)
+            plan.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish, bf16=args.bf16_out,
+                           consume=not args.keep_blocks and not args.no_finish)
 
     # warm-up: at least --warmup steps AND at least --min-warm-s seconds of back-to-back steps, so that the
     # timed steps see the clocks of a long run (the power cap pulls them down within about a second)
@@ -471,7 +472,8 @@ def run_ours(args):
                 if args.two_step:
                     pl.exec_opts(Ai, Bi, partials, Cs, bf16=args.bf16_out)
                 else:
-                    pl.exec_opts(Ai, Bi, partials, Cs, direct=True, finish=not args.no_finish, bf16=args.bf16_out)
+                    pl.exec_opts(Ai, Bi, partials, Cs, direct=True, finish=not args.no_finish, bf16=args.bf16_out,
+                                 consume=not args.keep_blocks and not args.no_finish)
                 pl.assemble(partials, Cs)
                 comp_done[i].record(s_comp)
             with torch.cuda.stream(s_out):
@@ -533,6 +535,8 @@ def run_ours(args):
         live = (t["flags"] & 1) == 0
         al, be, ka = (t["m1"] - t["m0"]).astype(np.float64), (t["n1"] - t["n0"]).astype(np.float64), (t["k1"] - t["k0"]).astype(np.float64)
         vbytes = float((((al + be) * ka * 2 + al * be * 4) * live).sum())
+        if not args.two_step:                          # every block into the arena (the timed steps use some up on arrival)
+            plan.exec_opts(A, B, partials, C, direct=True, finish=not args.no_finish, bf16=args.bf16_out)
         plan.verify(A, B, partials, seed=1)            # first call allocates
         v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         v0.record()
@@ -551,6 +555,7 @@ def run_ours(args):
         shared = dict(tensors=d_tensors)
         base = dict(opts)
         legs = [("same workload, two-step (cleave_exec + cleave_assemble of every GEMM)", args.config, args.scale, base, "two-step", False, shared),
+                ("same workload, every block kept in the arena", args.config, args.scale, base, "fused", False, dict(shared, consume=False)),
                 ("same workload, bf16 outputs", args.config, args.scale, base, "fused", True, shared)]
         if args.gran_m is None:
             legs.append(("same workload, row granule 256", args.config, args.scale, dict(base, gran_m=256), "fused", False, shared))
@@ -601,7 +606,8 @@ def run_ours(args):
             "parallelism": "replicas only" if world > 1 else "1 GPU",
             "write_out": ("two-step: every block to the arena, every GEMM through cleave_assemble" if args.two_step else
                           "in the exec kernel: one-slice blocks stored in C" +
-                          ("" if args.no_finish else ", K-split cells summed in fixed order by the block stored last")),
+                          ("" if args.no_finish else ", K-split cells summed in fixed order by the block that arrives last" +
+                           ("" if args.keep_blocks else " (that block is used up on arrival, the others are stored in the arena)"))),
             "c_dtype": "bf16" if args.bf16_out else "fp32",
             "gemms_finished_in_exec_kernel": int(sum(in_kernel)),
             "l2": "not flushed; operands + arena + outputs per step (~%.1f GB) far exceed the 126 MB L2" %
@@ -653,6 +659,8 @@ def main():
     ap.add_argument("--two-step", action="store_true", help="cleave_exec + full cleave_assemble instead of the fused write-out")
     ap.add_argument("--no-finish", action="store_true", help="fused write-out of one-slice GEMMs only; K-split GEMMs go through cleave_assemble")
     ap.add_argument("--gran-m", type=int, default=None, help="row granule of the planner (default 128)")
+    ap.add_argument("--keep-blocks", action="store_true", help="store every partial block in the arena (default: the block that "
+                    "completes a K-split cell is summed on arrival and not stored)")
     ap.add_argument("--bf16-out", action="store_true", help="C in bf16 (rounded from the fp32 sums) instead of fp32")
     ap.add_argument("--min-warm-s", type=float, default=1.5, help="warm up for at least this long before the timed steps")
     ap.add_argument("--no-other", action="store_true", help="skip the short legs on other modes and workloads")

@@ -197,6 +197,13 @@ CLEAVE_API int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const v
  *                       K-slices are cut into unequal blocks (after a memory repair), with more than
  *                       8 K-slices or with N % 4 != 0 are left to cleave_assemble; so is every GEMM
  *                       when a task is dropped, and after a cleave_reissue;
+ *   CLEAVE_EXEC_CONSUME (with FINISH) the block that completes a cell is used up on arrival: it is
+ *                       added to the other K-slices' blocks and never stored in the arena (a third
+ *                       less partial-block traffic for two K-slices).  Afterwards the arena holds
+ *                       S - 1 of a cell's S blocks, so cleave_verify (E_UNSUPPORTED) and
+ *                       cleave_reissue (E_INVAL) are refused until the next execution without it.  Ignored (every block is stored) when a task
+ *                       is dropped or superseded, because cleave_assemble will need every block.
+ *                       The sums and their bits are the same.
  *   CLEAVE_EXEC_BF16    C holds bf16: every value written to C, by this call and by the
  *                       cleave_assemble / cleave_reissue that follow it, is the fp32 value rounded to
  *                       nearest even (ld = N elements, 16-byte aligned).  Arena blocks stay fp32.
@@ -211,6 +218,7 @@ CLEAVE_API int cleave_exec_fused(cleave_plan_t* p, const void* const* A, const v
 #define CLEAVE_EXEC_DIRECT 1u
 #define CLEAVE_EXEC_FINISH 2u
 #define CLEAVE_EXEC_BF16   4u
+#define CLEAVE_EXEC_CONSUME 8u
 CLEAVE_API int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* B, float* partials,
                                 void* const* C, uint32_t flags, uint32_t level_begin, uint32_t level_end, void* stream);
 

@@ -5,7 +5,7 @@ binding only marshals arguments; every step runs in the library.  There is no fa
 use of anything but the `build` submodule loads the library and raises if it has not been built.
 """
 _BINDING_NAMES = ("CleaveError", "Plan", "default_opts", "lib", "lib_path", "plan", "plan_uniform",
-                  "GEMM_DTYPE", "TASK_DTYPE", "DEVICE_DTYPE", "strerror", "EXEC_DIRECT", "EXEC_FINISH", "EXEC_BF16")
+                  "GEMM_DTYPE", "TASK_DTYPE", "DEVICE_DTYPE", "strerror", "EXEC_DIRECT", "EXEC_FINISH", "EXEC_BF16", "EXEC_CONSUME")
 
 
 def __getattr__(name):

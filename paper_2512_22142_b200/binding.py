@@ -73,7 +73,7 @@ for _name, (_res, _args) in _sig.items():
     _f.restype, _f.argtypes = _res, _args
 
 
-EXEC_DIRECT, EXEC_FINISH, EXEC_BF16 = 1, 2, 4
+EXEC_DIRECT, EXEC_FINISH, EXEC_BF16, EXEC_CONSUME = 1, 2, 4, 8
 
 
 def strerror(code: int) -> str:
@@ -195,12 +195,13 @@ class Plan:
         _check(lib.cleave_exec_fused(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(), pc.ctypes.data,
                                      _stream(stream)), "cleave_exec_fused")
 
-    def exec_opts(self, A, B, partials, Cs=None, direct=False, finish=False, bf16=False, level_begin=0,
+    def exec_opts(self, A, B, partials, Cs=None, direct=False, finish=False, bf16=False, consume=False, level_begin=0,
                   level_end=0xFFFFFFFF, stream=None) -> None:
         """cleave_exec_opts: flags CLEAVE_EXEC_DIRECT / FINISH / BF16 and a range of DAG levels."""
         pa, pb = _ptr_array(A), _ptr_array(B)
         pc = _ptr_array(Cs) if Cs is not None else None
-        flags = (EXEC_DIRECT if direct else 0) | (EXEC_FINISH if finish else 0) | (EXEC_BF16 if bf16 else 0)
+        flags = (EXEC_DIRECT if direct else 0) | (EXEC_FINISH if finish else 0) | (EXEC_BF16 if bf16 else 0) | \
+            (EXEC_CONSUME if consume else 0)
         _check(lib.cleave_exec_opts(self._h, pa.ctypes.data, pb.ctypes.data, partials.data_ptr(),
                                     pc.ctypes.data if pc is not None else None, flags, level_begin, level_end,
                                     _stream(stream)), "cleave_exec_opts")

@@ -437,7 +437,8 @@ int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* 
                      uint32_t flags, uint32_t level_begin, uint32_t level_end, void* stream) {
     int rc = check_exec_args(p, A, B, partials);
     if (rc) return rc;
-    if (flags & ~(uint32_t)(CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH | CLEAVE_EXEC_BF16)) return CLEAVE_E_INVAL;
+    if (flags & ~(uint32_t)(CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH | CLEAVE_EXEC_BF16 | CLEAVE_EXEC_CONSUME)) return CLEAVE_E_INVAL;
+    if ((flags & CLEAVE_EXEC_CONSUME) && !(flags & CLEAVE_EXEC_FINISH)) return CLEAVE_E_INVAL;
     if ((flags & (CLEAVE_EXEC_DIRECT | CLEAVE_EXEC_FINISH)) && !C) return CLEAVE_E_INVAL;
     if (level_begin > level_end) return CLEAVE_E_INVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -446,7 +447,7 @@ int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* 
         if (level_begin != 0 || level_end < p->n_levels) return CLEAVE_E_UNSUPPORTED;
         try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
         p->mode = (flags & CLEAVE_EXEC_BF16) ? MODE_BF16 : 0u;
-        p->fused = p->finished = false;
+        p->fused = p->finished = p->consumed = false;
         p->out_bf16 = (p->mode & MODE_BF16) != 0;
         try { return run_tasks_plain(p, 0, true, A, B, partials, st); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     }
@@ -464,6 +465,10 @@ int cleave_exec_opts(cleave_plan_t* p, const void* const* A, const void* const* 
     for (size_t i = 0; whole && i < p->tasks.size(); ++i)
         if (p->dropped[i] || (p->tasks[i].flags & CLEAVE_TASK_SUPERSEDED)) whole = false;   // replacement pieces join no cell
     p->finished = (p->mode & MODE_FINISH) && whole;
+    // blocks are only used up on arrival when every cell is going to be summed in this launch: with a task
+    // missing, cleave_assemble needs them all
+    p->consumed = p->finished && (flags & CLEAVE_EXEC_CONSUME);
+    if (p->consumed) p->mode |= MODE_CONSUME;
     return run_tiles(p, 0, (uint32_t)p->tiles.size(), true, level_begin, level_end, partials, st);
 }
 
@@ -513,6 +518,7 @@ int cleave_reissue(cleave_plan_t* p, const uint32_t* failed, uint32_t n, const v
     int rc = check_exec_args(p, A, B, partials);
     if (rc) return rc;
     if (n && !failed) return CLEAVE_E_INVAL;
+    if (p->consumed) return CLEAVE_E_INVAL;            // the arena lacks the blocks that were used up: execute again first
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     try {
         RC_TRY(sync_device_state(p, st));
@@ -568,6 +574,7 @@ int cleave_verify(cleave_plan_t* p, const void* const* A, const void* const* B, 
     if (!p || !A || !B || !partials || !n_bad || !(tol >= 0.f)) return CLEAVE_E_INVAL;
     for (const auto& g : p->gemms) if ((g.K % 4) || (g.lda % 8) || (g.ldb % 8)) return CLEAVE_E_UNSUPPORTED;
     if (p->fused && p->out_bf16) return CLEAVE_E_UNSUPPORTED;      // blocks written to C as bf16 are not checked
+    if (p->consumed) return CLEAVE_E_UNSUPPORTED;                   // blocks used up on arrival are not in the arena
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     try { RC_TRY(sync_device_state(p, st)); } catch (const std::bad_alloc&) { return CLEAVE_E_NOMEM; }
     DeviceState* d = p->dev;

@@ -30,7 +30,8 @@
 // Usually a strip already finds every other slice's block stored when its tile is handed out (a GEMM is
 // walked K-range by K-range): it then asks for those blocks to be brought into L2 while its own MMAs
 // still run, and adds them to its accumulator values on their way out (no second pass over its own
-// block).  A strip that only turns out to be last after storing its block reads all blocks back.
+// block; under MODE_CONSUME it does not even store that block: it is used up on arrival).  A strip that
+// only turns out to be last after storing its block reads all blocks back.
 // Under MODE_BF16 values written to C are rounded to bf16.
 //
 // DAG levels: tiles are ordered by level, and before the scheduler hands out the first tile of a
@@ -274,6 +275,7 @@ struct SummedChunk {
     uint32_t ldc;
     uint32_t taddr;             // tensor-memory address of the chunk
     bool last_chunk;            // reading it frees the accumulator slot
+    bool keep_own;              // the own block is stored in the arena as well
     uint32_t acc_empty_leader;
 };
 template <int SP, bool BF16>
@@ -323,7 +325,7 @@ __device__ __forceinline__ void summed_chunk(const SummedChunk& k, float* stage_
             const uint32_t r = rr + 4u * (uint32_t)(b + x);
             if (r >= rows_here) continue;
             const float4 own = staged_f4(stage_tile, r, lane & 7u);
-            *reinterpret_cast<float4*>(k.own_blk + (uint64_t)r * k.own_ld + k.c0 + cc) = own;
+            if (k.keep_own) *reinterpret_cast<float4*>(k.own_blk + (uint64_t)r * k.own_ld + k.c0 + cc) = own;
             float4 v[SP];
 #pragma unroll
             for (int s = 0; s < SP; ++s) {
@@ -598,7 +600,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     k.own_blk = P.partials + sg.out_off + (uint64_t)row0 * sg.ld; k.own_ld = sg.ld;
                     k.row0 = row0; k.rows_here = rows_here; k.c0 = c0; k.cols = width[q];
                     k.c_base = P.c_ptrs[gemm]; k.c_off = c_off + (q ? split : 0u); k.ldc = ldc;
-                    k.taddr = taddr + ct; k.last_chunk = (c + 1 == nchunk); k.acc_empty_leader = acc_empty_leader;
+                    k.taddr = taddr + ct; k.last_chunk = (c + 1 == nchunk); k.keep_own = !(P.mode & MODE_CONSUME); k.acc_empty_leader = acc_empty_leader;
                     if (nslices <= 2) { if (out_bf16) summed_chunk<2, true>(k, stage_tile, lane); else summed_chunk<2, false>(k, stage_tile, lane); }
                     else if (nslices <= 4) { if (out_bf16) summed_chunk<4, true>(k, stage_tile, lane); else summed_chunk<4, false>(k, stage_tile, lane); }
                     else { if (out_bf16) summed_chunk<8, true>(k, stage_tile, lane); else summed_chunk<8, false>(k, stage_tile, lane); }

@@ -58,7 +58,9 @@ enum : uint32_t { TILE_LIVE0 = 1u, TILE_LIVE1 = 2u, TILE_END = 4u, TILE_A_MN = 8
 //   FINISH  in a GEMM with several K-slices the last block of a cell to arrive sums the cell's blocks
 //           (all of them are in the arena by then) in the fixed tree order and writes C
 //   BF16    C holds bf16 (round to nearest even from the fp32 value) instead of fp32
-enum : uint32_t { MODE_DIRECT = 1u, MODE_FINISH = 2u, MODE_BF16 = 4u };
+//   CONSUME (with FINISH) a block that completes its cell when its tile is handed out is summed on arrival and not
+//           stored in the arena
+enum : uint32_t { MODE_DIRECT = 1u, MODE_FINISH = 2u, MODE_BF16 = 4u, MODE_CONSUME = 8u };
 
 // Partial block of one K-slice inside a cell of the in-kernel sum.
 struct FinRef {
@@ -122,6 +124,7 @@ struct cleave_plan_s {
     bool fused = false;                            // last execution wrote one-slice GEMMs straight to C
     bool finished = false;                         // ... and summed every cell of the finishable GEMMs itself, none missing
     bool out_bf16 = false;                         // ... into bf16 outputs
+    bool consumed = false;                         // ... without storing the blocks that completed their cells
     uint64_t wait_limit_ns = 2000000000ull;        // bound of every device-side wait
 
     cleave::DeviceState* dev = nullptr;

@@ -44,6 +44,14 @@ def test_config3_sampled_entries_and_freivalds():
     _check_against_oracle(w, ts, run)
     bad, vals = p.verify(run.A, run.B, run.partials, seed=5)     # every returned block passes the vector check
     assert bad == 0 and np.all(np.abs(vals[:, 0] - vals[:, 1]) <= 5e-6 * vals[:, 2] + 1e-5)
+    # the mode the benchmark times (blocks that complete a cell are used up on arrival): the same bits
+    keep = [c.clone() for c in run.C]
+    for c in run.C:
+        c.fill_(float("nan"))
+    run.exec_opts(direct=True, finish=True, consume=True); run.assemble(); p.check_status()
+    torch.cuda.synchronize()
+    for g, a, b in zip(w.gemms, keep, run.C):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32)), g.name
 
 
 def test_config4_churn_full_size():

@@ -43,6 +43,54 @@ def test_in_kernel_sum_of_k_split_cells_is_bit_identical(opts):
     assert all(done[i] == p.task_num_tiles(i) for i in range(p.num_tasks))
 
 
+def test_blocks_used_up_on_arrival():
+    """CLEAVE_EXEC_CONSUME: the block that completes a cell is added to the others on its way out and
+    never stored -- same bits in C, one block per cell missing from the arena; with a task dropped the
+    flag is ignored and the usual recovery works."""
+    import paper_2512_22142_b200 as cl
+    w = ci.config(4, 8)
+    ts = ci.make_tensors(w)
+    opts = dict(kslice_max=512)
+    good = _two_step(w, ts, **opts)
+    p = lib_plan_for(w, **opts)
+    run = GpuRun(w, ts, p)
+    run.exec_opts(direct=True, finish=True, consume=True); run.assemble(); p.check_status()
+    assert p.num_launches == 5
+    for g, a, b in zip(w.gemms, good, run.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), g.name
+    # the arena started as NaN: in every cell of a K-split GEMM at most one slice's block is missing (the one
+    # that completed the cell; which strips find their cell complete on arrival depends on timing)
+    t = p.tasks()
+    arena = run.partials.cpu().numpy()
+    for gi, g in enumerate(w.gemms):
+        if p.ksplit(gi) == 1:
+            continue
+        missing = np.zeros((g.M, g.N), dtype=np.int32)
+        for x in t[t["gemm"] == gi]:
+            a_, b_ = int(x["m1"] - x["m0"]), int(x["n1"] - x["n0"])
+            blk = arena[int(x["part_off"]):int(x["part_off"]) + a_ * b_].reshape(a_, b_)
+            missing[int(x["m0"]):int(x["m1"]), int(x["n0"]):int(x["n1"])] += np.isnan(blk)
+        assert missing.max() <= 1, g.name
+    with pytest.raises(cl.CleaveError) as e:
+        p.verify(run.A, run.B, run.partials, seed=1)
+    assert e.value.code == -2
+    with pytest.raises(cl.CleaveError) as e:
+        run.reissue([0])
+    assert e.value.code == -1
+    # a dropped task: every block that runs is stored, the assembly kernel sums after the reissue
+    failed = ci.make_failed_ids(p.num_tasks, w.fail_frac, w.seed + 2)
+    p.set_drops(failed)
+    run.partials.fill_(float("nan"))
+    for c in run.C:
+        c.fill_(float("nan"))
+    run.exec_opts(direct=True, finish=True, consume=True); run.assemble()
+    assert p.status() == -9
+    run.reissue(failed); run.assemble()
+    assert p.status() == 0
+    for g, a, b in zip(w.gemms, good, run.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), g.name
+
+
 def test_unequal_slices_fall_back_to_the_assembly_kernel():
     """Blocks off the 128-grid (granule 64) under memory budgets so small that the K-slices of a block
     are repaired into different pieces: such a GEMM cannot be summed cell by cell in the exec kernel
