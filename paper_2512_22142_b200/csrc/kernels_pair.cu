@@ -73,6 +73,12 @@ __device__ __forceinline__ void cluster_arrive_wait() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same for arrivals that only say "I have read it" (a ring slot, an accumulator slot): nothing this
+// thread wrote has to be seen by the waiting side, so the arrival must not wait for the thread's global
+// stores in flight, which a cluster-scope release does (about a thousand cycles behind a burst of stores).
+__device__ __forceinline__ void mbar_arrive_cluster_read_done(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait_cl(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -312,7 +318,7 @@ __device__ __forceinline__ void summed_chunk(const SummedChunk& k, float* stage_
         if (k.last_chunk) {                                  // slot fully read: hand it back to the leader
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(k.acc_empty_leader);
+            if (lane == 0) mbar_arrive_cluster_read_done(k.acc_empty_leader);
         }
         stage_row(stage_tile, lane, v);
     }
@@ -376,8 +382,8 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
         if (rank == 0 && lane == 0) {
             uint32_t levels_done = 0;                  // every level below this one is known to be complete
             for (uint32_t i = 0;; ++i) {
-                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-                if (!mbar_wait_cl(smem_u32(&sh.sched_empty[q]), par ^ 1u, W)) break;
+                // The next live tile is fetched (ticket, then its descriptor: two dependent trips to L2) BEFORE
+                // waiting for a free slot: the wait normally lasts longer than the fetch, which so costs nothing.
                 uint4 w[kTileWords16];
                 bool end = false;
                 for (;;) {
@@ -388,6 +394,8 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     for (int x = 0; x < kTileWords16; ++x) w[x] = __ldg(src + x);
                     if (w[0].y & (TILE_LIVE0 | TILE_LIVE1)) break;      // TileDesc::flags
                 }
+                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+                if (!mbar_wait_cl(smem_u32(&sh.sched_empty[q]), par ^ 1u, W)) break;
                 if (end) {
 #pragma unroll
                     for (int x = 0; x < kTileWords16; ++x) w[x] = make_uint4(0, 0, 0, 0);
@@ -423,7 +431,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             const uint32_t rows0 = (flags & TILE_LIVE0) ? sl.h[0].rows : 0u, rows1 = (flags & TILE_LIVE1) ? sl.h[1].rows : 0u;
             const uint32_t a_x = sl.h[rank].m_row;
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
+            if (lane == 0) mbar_arrive_cluster_read_done(sched_empty_leader0 + q * 8u);
             if (flags & TILE_END) break;
             const CUtensorMap* map_a = P.maps + kMapsPerGemm * gemm;
             const CUtensorMap* map_b = map_a + 1;
@@ -530,35 +538,61 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
         const uint32_t acc_empty_leader = mapa_shared(smem_u32(&sh.acc_empty[group]), 0u);
         const bool out_bf16 = P.mode & MODE_BF16;
         uint32_t used = 0, tile_no = 0;
+        // Bookkeeping owed for strips already stored: lane j keeps entry j (the quadrants' tasks, the level and
+        // how many strips to count off it).  The counts may only be made after a fence that waits for the
+        // strip's stores, and such a fence costs thousands of cycles behind a burst of stores; so it is paid
+        // when the warp would wait anyway (no tile ready), when kMaxOwed entries have gathered, before any
+        // bookkeeping that cannot wait (cells of the in-kernel sum), and when the warp leaves.
+        constexpr uint32_t kMaxOwed = 8;
+        uint32_t owed = 0, owed_task0 = 0xFFFFFFFFu, owed_task1 = 0xFFFFFFFFu, owed_level = 0, owed_strips = 0;
+        auto count_owed = [&]() {                         // (the caller has fenced and synchronised the warp)
+            if (lane < owed) {
+                if (owed_task0 != 0xFFFFFFFFu) atomicAdd(&P.done[owed_task0], 1u);   // one count per warp and quadrant
+                if (owed_task1 != 0xFFFFFFFFu) atomicAdd(&P.done[owed_task1], 1u);
+                if (owed_strips) atomicSub(&P.level_left[owed_level], owed_strips);
+            }
+            owed = 0;
+            __syncwarp();
+        };
+        auto settle = [&]() {
+            if (owed) { __threadfence(); __syncwarp(); count_owed(); }
+        };
         for (uint32_t i = 0;; ++i) {
             const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-            bool ok = mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, W);
-            if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            bool ok = mbar_try_wait_cl(smem_u32(&sh.sched_full[q]), par);
+            if (!__all_sync(0xFFFFFFFFu, ok)) {
+                settle();
+                ok = mbar_wait_cl(smem_u32(&sh.sched_full[q]), par, W);
+                if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            }
             const TileDesc& sl = sh.slot[q];
             const uint32_t flags = sl.flags, gemm = sl.gemm, n_mma = sl.n_mma & 0xFFFFu, cols = sl.n_mma >> 16;
             const uint32_t level = sl.level & 0xFFFFu, nslices = (sl.level >> 16) & 0xFFu, kslice = sl.level >> 24;
             const uint32_t ldc = sl.ldc, n_col = sl.n_col, split = sl.split;
-            const TileHalf h = sl.h[rank];
+            // (the two column segments in variables of their own: an array indexed by the chunk's segment would live
+            // in local memory, and a local load queues behind the stores in flight)
+            const uint32_t h_m_row = sl.h[rank].m_row, h_rows = sl.h[rank].rows;
+            const TileSeg seg0 = sl.h[rank].seg[0], seg1 = sl.h[rank].seg[1];
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(sched_empty_leader0 + q * 8u);
+            if (lane == 0) mbar_arrive_cluster_read_done(sched_empty_leader0 + q * 8u);
             if (flags & TILE_END) break;
             const bool mine = (tile_no & 1u) == group;       // tiles alternate between the two accumulator slots
             ++tile_no;
             if (!mine) continue;
-            const uint32_t rows = (flags & (TILE_LIVE0 << rank)) ? h.rows : 0u;
+            const uint32_t rows = (flags & (TILE_LIVE0 << rank)) ? h_rows : 0u;
             const uint32_t rows_here = rows > quad * 32u ? min(32u, rows - quad * 32u) : 0u;
             const uint32_t row0 = quad * 32u;
             // a block of a one-slice GEMM is final: it may go straight to its place in C
             const bool direct = (P.mode & MODE_DIRECT) && (flags & TILE_SINGLE);
             const bool to_bf16 = direct && out_bf16;
-            const uint64_t c_off = (uint64_t)h.m_row * ldc + n_col;            // the half-tile's (0, 0) in C
+            const uint64_t c_off = (uint64_t)h_m_row * ldc + n_col;            // the half-tile's (0, 0) in C
             // the one or two column segments of the half-tile: quadrants of possibly different tasks
             const uint32_t width[2] = {min(split, cols), cols > split ? cols - split : 0u};
             bool cell[2], sum_now[2] = {false, false};
             const FinRef* refs[2] = {nullptr, nullptr};
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                const TileSeg& sg = h.seg[q];
+                const TileSeg& sg = q ? seg1 : seg0;
                 cell[q] = rows && sg.live && width[q] && (P.mode & MODE_FINISH) && !direct && sg.fin != kNoFin;
                 // Is every other K-slice's block of this strip's cell stored already?  Then this strip is the last
                 // one: start bringing those blocks into L2 now, while the MMAs of this tile still run.
@@ -581,24 +615,29 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     }
                 }
             }
-            ok = mbar_wait_cl(smem_u32(&sh.acc_full[group]), used & 1u, W);
-            if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            ok = mbar_try_wait_cl(smem_u32(&sh.acc_full[group]), used & 1u);
+            if (!__all_sync(0xFFFFFFFFu, ok)) {
+                settle();
+                ok = mbar_wait_cl(smem_u32(&sh.acc_full[group]), used & 1u, W);
+                if (!__all_sync(0xFFFFFFFFu, ok)) break;
+            }
             ++used;
             tc_fence_after();
             const uint32_t taddr = tmem_base + group * kAccCols + ((quad * 32u) << 16);
             const uint32_t nchunk = (n_mma + 31u) / 32u;
             for (uint32_t c = 0; c < nchunk; ++c) {
-                const uint32_t q = (c * 32u >= split) ? 1u : 0u;             // (split is a multiple of 32 when a second segment exists)
-                const TileSeg& sg = h.seg[q];
-                const bool live_chunk = rows_here && sg.live && c * 32u < cols;   // warp-uniform
+                const bool q = c * 32u >= split;             // (split is a multiple of 32 when a second segment exists)
+                const uint32_t sg_ld = q ? seg1.ld : seg0.ld, sg_live = q ? seg1.live : seg0.live;
+                const uint64_t sg_out_off = q ? seg1.out_off : seg0.out_off;
+                const bool live_chunk = rows_here && sg_live && c * 32u < cols;   // warp-uniform
                 const uint32_t ct = c * 32u;                 // chunk's first column in the half-tile ...
                 const uint32_t c0 = ct - (q ? split : 0u);   // ... and in its quadrant
-                if (live_chunk && sum_now[q]) {
+                if (live_chunk && (q ? sum_now[1] : sum_now[0])) {
                     // (cells exist only where float4 accesses are aligned and columns come in fours)
                     SummedChunk k;
-                    k.refs = refs[q]; k.nslices = nslices; k.mine = kslice; k.partials = P.partials;
-                    k.own_blk = P.partials + sg.out_off + (uint64_t)row0 * sg.ld; k.own_ld = sg.ld;
-                    k.row0 = row0; k.rows_here = rows_here; k.c0 = c0; k.cols = width[q];
+                    k.refs = q ? refs[1] : refs[0]; k.nslices = nslices; k.mine = kslice; k.partials = P.partials;
+                    k.own_blk = P.partials + sg_out_off + (uint64_t)row0 * sg_ld; k.own_ld = sg_ld;
+                    k.row0 = row0; k.rows_here = rows_here; k.c0 = c0; k.cols = q ? width[1] : width[0];
                     k.c_base = P.c_ptrs[gemm]; k.c_off = c_off + (q ? split : 0u); k.ldc = ldc;
                     k.taddr = taddr + ct; k.last_chunk = (c + 1 == nchunk); k.keep_own = !(P.mode & MODE_CONSUME); k.acc_empty_leader = acc_empty_leader;
                     if (nslices <= 2) { if (out_bf16) summed_chunk<2, true>(k, stage_tile, lane); else summed_chunk<2, false>(k, stage_tile, lane); }
@@ -612,13 +651,13 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 if (c + 1 == nchunk) {                       // slot fully read: hand it back to the leader
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+                    if (lane == 0) mbar_arrive_cluster_read_done(acc_empty_leader);
                 }
                 if (!live_chunk) continue;
                 stage_row(stage_tile, lane, v);
                 __syncwarp();
-                const uint32_t ld = direct ? ldc : sg.ld;
-                const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg.out_off + (uint64_t)row0 * sg.ld + c0;
+                const uint32_t ld = direct ? ldc : sg_ld;
+                const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg_out_off + (uint64_t)row0 * sg_ld + c0;
                 float* out_f32 = (direct ? static_cast<float*>(P.c_ptrs[gemm]) : P.partials) + out_off;
                 __nv_bfloat16* out_b16 = static_cast<__nv_bfloat16*>(P.c_ptrs[gemm]) + out_off;
                 const bool vec_ok = ((ld & 3u) == 0u) && ((out_off & 3ull) == 0ull);
@@ -644,14 +683,24 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 __syncwarp();
             }
             if (rows) {
+                const bool live0 = seg0.live && width[0], live1 = seg1.live && width[1];
+                const uint32_t n_live = (live0 ? 1u : 0u) + (live1 ? 1u : 0u);
+                if (!cell[0] && !cell[1]) {
+                    // nobody waits for these counts right now: owe them (see above)
+                    if (lane == owed) {
+                        owed_task0 = live0 ? seg0.task : 0xFFFFFFFFu; owed_task1 = live1 ? seg1.task : 0xFFFFFFFFu;
+                        owed_level = level; owed_strips = n_live;
+                    }
+                    if (++owed == kMaxOwed) settle();
+                    continue;
+                }
                 __threadfence();                             // this strip's stores before its arrival is counted
                 __syncwarp();
-                uint32_t n_live = 0;
+                count_owed();                                // (the fence covered the older strips' stores as well)
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
-                    const TileSeg& sg = h.seg[q];
+                    const TileSeg& sg = q ? seg1 : seg0;
                     if (!sg.live || !width[q]) continue;
-                    ++n_live;
                     if (lane == 0) atomicAdd(&P.done[sg.task], 1u);   // one count per warp and quadrant
                     if (!cell[q]) continue;
                     unsigned int before = 0;
@@ -679,6 +728,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 if (lane == 0 && n_live) atomicSub(&P.level_left[level], n_live);   // after everything this strip had to write
             }
         }
+        settle();                                            // whatever is still owed, also when the pair gives up
     }
 
     __syncwarp();
