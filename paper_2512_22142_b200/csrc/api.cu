@@ -25,6 +25,7 @@ struct DeviceState {
     uint32_t* failed_ids = nullptr;
     unsigned int* words = nullptr;    // [0] ticket, [1] status, [2] failed count
     CUtensorMap* maps = nullptr;
+    CUtensorMap* c_maps = nullptr;    // per GEMM: C as an fp32 matrix, 32 x 32 boxes (the exec kernel's bulk stores)
     AsmItem* asm_items = nullptr;
     AsmRef* asm_refs = nullptr;
     void** c_ptrs = nullptr;
@@ -95,6 +96,21 @@ int encode_map_groups(CUtensorMap* out, const void* base, uint64_t rows, uint64_
     return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
 }
 
+// fp32 tensor map over a row-major [rows x cols] matrix C: boxes of 32 x 32 elements (128-byte rows,
+// 128-byte swizzle): what an epilogue warp of the exec kernel stores with one bulk operation.
+int encode_c_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return CLEAVE_E_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
+}
+
 template <typename T>
 int dev_alloc(T** p, size_t n) {
     if (n == 0) n = 1;
@@ -119,6 +135,7 @@ int create_device_state(cleave_plan_s* p, cudaStream_t st, DeviceState* d) {
     RC_TRY(dev_alloc(&d->words, 4));
     CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
     RC_TRY(dev_alloc(&d->maps, kMapsPerGemm * ng));
+    RC_TRY(dev_alloc(&d->c_maps, ng));
     RC_TRY(dev_alloc(&d->c_ptrs, ng));
     RC_TRY(dev_alloc(&d->ldcs, ng));
     std::vector<uint32_t> ldc;
@@ -238,6 +255,14 @@ int upload_c_ptrs(cleave_plan_s* p, void* const* C, cudaStream_t st) {
     if (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin())) {
         d->last_c.assign(C, C + n);
         CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(void*), cudaMemcpyHostToDevice, st));
+        // fp32 views of the outputs for bulk stores (the kernel uses one only for fp32 output with N % 4 == 0)
+        std::vector<CUtensorMap> host(n);
+        for (size_t i = 0; i < n; ++i) {
+            const cleave_gemm_t& g = p->gemms[i];
+            if (g.N % 4 == 0) RC_TRY(encode_c_map(&host[i], C[i], g.M, g.N));
+            else std::memset(&host[i], 0, sizeof(CUtensorMap));
+        }
+        CU_TRY(cudaMemcpyAsync(d->c_maps, host.data(), n * sizeof(CUtensorMap), cudaMemcpyHostToDevice, st));
     }
     return 0;
 }
@@ -259,7 +284,7 @@ int run_tiles(cleave_plan_s* p, uint32_t tile_begin, uint32_t tile_end, bool fre
         // one cluster of two CTAs per pair of SMs, never more clusters than tiles
         const uint32_t clusters = std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)d->sm_count / 2, tile_end - tile_begin));
         ExecParams e;
-        e.tiles = d->tiles; e.tile_end = tile_end; e.ticket = d->words + 0; e.maps = d->maps; e.partials = partials;
+        e.tiles = d->tiles; e.tile_end = tile_end; e.ticket = d->words + 0; e.maps = d->maps; e.c_maps = d->c_maps; e.partials = partials;
         e.c_ptrs = d->c_ptrs; e.done = d->done; e.status = d->words + 1;
         e.fin_ref0 = d->fin_ref0; e.fin_refs = d->fin_refs; e.fin_count = d->fin_count; e.level_left = d->level_left;
         e.mode = p->mode; e.wait_limit_ns = p->wait_limit_ns;
@@ -318,7 +343,7 @@ int status_to_code(unsigned int s) {
 void device_state_free(DeviceState* d) {
     if (!d) return;
     cudaFree(d->tasks); cudaFree(d->tiles); cudaFree(d->dropped); cudaFree(d->done); cudaFree(d->ntiles);
-    cudaFree(d->failed_ids); cudaFree(d->words); cudaFree(d->maps); cudaFree(d->asm_items); cudaFree(d->asm_refs);
+    cudaFree(d->failed_ids); cudaFree(d->words); cudaFree(d->maps); cudaFree(d->c_maps); cudaFree(d->asm_items); cudaFree(d->asm_refs);
     cudaFree(d->c_ptrs); cudaFree(d->ldcs); cudaFree(d->fin_ref0); cudaFree(d->fin_refs); cudaFree(d->fin_count);
     cudaFree(d->level_left); cudaFree(d->gemm_table); cudaFree(d->ksplit_table); cudaFree(d->ab_ptrs);
     cudaFree(d->verify_out);

@@ -145,6 +145,14 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const void* tmap,
         "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// Bulk store of a 32 x 32 fp32 box from this CTA's shared memory (rows of 128 bytes, 128-byte swizzle) into a
+// matrix in this GPU's memory; completion is tracked by the issuing thread's bulk groups.
+__device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int32_t c0, int32_t c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tmap), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }   // sources may be reused
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }             // the stores are complete
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -286,7 +294,7 @@ struct SummedChunk {
 };
 template <int SP, bool BF16>
 __device__ __forceinline__ void summed_chunk(const SummedChunk& k, float* stage_tile, uint32_t lane) {
-    constexpr int RB = SP <= 2 ? 8 : (SP <= 4 ? 4 : 2);      // rows per lane whose loads are in flight together
+    constexpr int RB = SP <= 2 ? 8 : (SP <= 4 ? 4 : 1);      // rows per lane whose loads are in flight together
     constexpr int NO = SP - 1;                               // other slices (slot j holds slice j, or j + 1 from `mine` on)
     const uint32_t rr = lane >> 3, cc = (lane & 7u) * 4u;
     const uint32_t rows_here = (k.c0 + cc >= k.cols) ? 0u : k.rows_here;   // ragged last chunk (columns come in fours)
@@ -554,8 +562,21 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             owed = 0;
             __syncwarp();
         };
+        // Blocks that go straight to an fp32 C leave as bulk stores of whole 32 x 32 chunks (issued by lane 0, which
+        // then does not wait for them): `bulk_reading` = a store may still be reading the staging tile,
+        // `bulk_flying` = stores of this warp may be incomplete (they must be complete before anything is counted).
+        bool bulk_reading = false, bulk_flying = false;
+        uint32_t c_map_gemm = 0xFFFFFFFFu;
+        auto staging_free = [&]() {
+            if (bulk_reading) { if (lane == 0) bulk_wait_read_all(); __syncwarp(); bulk_reading = false; }
+        };
+        auto fence_stores = [&]() {                       // every store of this warp so far, plain or bulk, is visible
+            if (bulk_flying) { if (lane == 0) bulk_wait_all(); __syncwarp(); bulk_flying = bulk_reading = false; }
+            __threadfence();
+            __syncwarp();
+        };
         auto settle = [&]() {
-            if (owed) { __threadfence(); __syncwarp(); count_owed(); }
+            if (owed) { fence_stores(); count_owed(); }
         };
         for (uint32_t i = 0;; ++i) {
             const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
@@ -585,6 +606,11 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             // a block of a one-slice GEMM is final: it may go straight to its place in C
             const bool direct = (P.mode & MODE_DIRECT) && (flags & TILE_SINGLE);
             const bool to_bf16 = direct && out_bf16;
+            const bool bulk_ok = direct && !out_bf16 && rows_here == 32u && ((ldc | n_col) & 3u) == 0u;
+            if (bulk_ok && gemm != c_map_gemm) {
+                if (lane == 0) tensormap_acquire(P.c_maps + gemm);
+                c_map_gemm = gemm;
+            }
             const uint64_t c_off = (uint64_t)h_m_row * ldc + n_col;            // the half-tile's (0, 0) in C
             // the one or two column segments of the half-tile: quadrants of possibly different tasks
             const uint32_t width[2] = {min(split, cols), cols > split ? cols - split : 0u};
@@ -633,6 +659,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 const uint32_t ct = c * 32u;                 // chunk's first column in the half-tile ...
                 const uint32_t c0 = ct - (q ? split : 0u);   // ... and in its quadrant
                 if (live_chunk && (q ? sum_now[1] : sum_now[0])) {
+                    staging_free();
                     // (cells exist only where float4 accesses are aligned and columns come in fours)
                     SummedChunk k;
                     k.refs = q ? refs[1] : refs[0]; k.nslices = nslices; k.mine = kslice; k.partials = P.partials;
@@ -654,7 +681,18 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     if (lane == 0) mbar_arrive_cluster_read_done(acc_empty_leader);
                 }
                 if (!live_chunk) continue;
+                staging_free();
                 stage_row(stage_tile, lane, v);
+                if (bulk_ok && ct + 32u <= cols) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the staged values, before the bulk store reads them
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(P.c_maps + gemm, smem_u32(stage_tile), (int32_t)(n_col + ct), (int32_t)(h_m_row + row0));
+                        bulk_commit();
+                    }
+                    bulk_reading = bulk_flying = true;
+                    continue;
+                }
                 __syncwarp();
                 const uint32_t ld = direct ? ldc : sg_ld;
                 const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg_out_off + (uint64_t)row0 * sg_ld + c0;
@@ -694,8 +732,7 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                     if (++owed == kMaxOwed) settle();
                     continue;
                 }
-                __threadfence();                             // this strip's stores before its arrival is counted
-                __syncwarp();
+                fence_stores();                              // this strip's stores before its arrival is counted
                 count_owed();                                // (the fence covered the older strips' stores as well)
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
