@@ -386,42 +386,63 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
     const uint32_t tmem_base = sh.tmem_base;
 
     if (warp == kSchedWarp) {
-        // ---- scheduler (leader only): ticket -> descriptor -> both CTAs' slot rings -----------------------
-        if (rank == 0 && lane == 0) {
+        // ---- scheduler (leader only): tickets -> descriptors -> both CTAs' slot rings ----------------------------
+        // A fetch is two dependent trips to L2 (the ticket, then the descriptor), a few thousand cycles behind a
+        // burst of stores: too long for pairs that run a handful of K-blocks.  So after such a pair the next
+        // fetch takes four tickets with one atomic and lane b loads descriptor b, all at once; the lanes
+        // then publish in ticket order.  Longer pairs are fetched one by one (a cluster that holds several of
+        // them would keep the others waiting at the end of the list, or of a small GEMM's share of it).
+        if (rank == 0) {
             uint32_t levels_done = 0;                  // every level below this one is known to be complete
-            for (uint32_t i = 0;; ++i) {
-                // The next live tile is fetched (ticket, then its descriptor: two dependent trips to L2) BEFORE
-                // waiting for a free slot: the wait normally lasts longer than the fetch, which so costs nothing.
+            uint32_t i = 0;                            // slots published so far
+            uint32_t batch = 1;
+            bool stop = false;
+            while (!stop) {
+                uint32_t t0 = 0;
+                if (lane == 0) t0 = atomicAdd(P.ticket, batch);
+                t0 = __shfl_sync(0xFFFFFFFFu, t0, 0);
+                const uint32_t t = t0 + lane;
                 uint4 w[kTileWords16];
-                bool end = false;
-                for (;;) {
-                    const uint32_t t = atomicAdd(P.ticket, 1u);
-                    if (t >= P.tile_end) { end = true; break; }
+                if (lane < batch && t < P.tile_end) {
                     const uint4* src = reinterpret_cast<const uint4*>(P.tiles + t);
 #pragma unroll
                     for (int x = 0; x < kTileWords16; ++x) w[x] = __ldg(src + x);
-                    if (w[0].y & (TILE_LIVE0 | TILE_LIVE1)) break;      // TileDesc::flags
-                }
-                const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
-                if (!mbar_wait_cl(smem_u32(&sh.sched_empty[q]), par ^ 1u, W)) break;
-                if (end) {
+                } else {
 #pragma unroll
                     for (int x = 0; x < kTileWords16; ++x) w[x] = make_uint4(0, 0, 0, 0);
                     w[0].y = TILE_END;
-                } else {
-                    // a tile of a higher DAG level runs only after every strip of the lower levels is written
-                    const uint32_t level = w[1].w & 0xFFFFu;         // TileDesc::level
-                    bool ok = true;
-                    while (ok && levels_done < level) { ok = wait_zero(P.level_left + levels_done, W); if (ok) ++levels_done; }
-                    if (!ok) break;
                 }
-                uint4* dst = reinterpret_cast<uint4*>(&sh.slot[q]);
-                const uint32_t peer_slot = mapa_shared(smem_u32(&sh.slot[q]), 1u);
+                uint32_t next_batch = 1;
+                for (uint32_t b = 0; b < batch && !stop; ++b) {
+                    uint32_t action = 0;               // 0 nothing to run in this pair, 1 published, 2 end of the list published, 3 gave up
+                    if (lane == b && (w[0].y & (TILE_LIVE0 | TILE_LIVE1 | TILE_END))) {      // TileDesc::flags
+                        const uint32_t q = i % kSchedSlots, par = (i / kSchedSlots) & 1u;
+                        bool ok = mbar_wait_cl(smem_u32(&sh.sched_empty[q]), par ^ 1u, W);
+                        if (ok && !(w[0].y & TILE_END)) {
+                            // a tile of a higher DAG level runs only after every strip of the lower levels is written
+                            const uint32_t level = w[1].w & 0xFFFFu;         // TileDesc::level
+                            while (ok && levels_done < level) { ok = wait_zero(P.level_left + levels_done, W); if (ok) ++levels_done; }
+                        }
+                        if (ok) {
+                            uint4* dst = reinterpret_cast<uint4*>(&sh.slot[q]);
+                            const uint32_t peer_slot = mapa_shared(smem_u32(&sh.slot[q]), 1u);
 #pragma unroll
-                for (int x = 0; x < kTileWords16; ++x) { dst[x] = w[x]; st_shared_cluster_v4(peer_slot + 16 * x, w[x]); }
-                mbar_arrive_cluster(mapa_shared(smem_u32(&sh.sched_full[q]), 0u));
-                mbar_arrive_cluster(mapa_shared(smem_u32(&sh.sched_full[q]), 1u));
-                if (end) break;
+                            for (int x = 0; x < kTileWords16; ++x) { dst[x] = w[x]; st_shared_cluster_v4(peer_slot + 16 * x, w[x]); }
+                            mbar_arrive_cluster(mapa_shared(smem_u32(&sh.sched_full[q]), 0u));
+                            mbar_arrive_cluster(mapa_shared(smem_u32(&sh.sched_full[q]), 1u));
+                        }
+                        action = !ok ? 3u : ((w[0].y & TILE_END) ? 2u : 1u);
+                    }
+                    action = __shfl_sync(0xFFFFFFFFu, action, b);
+                    levels_done = __shfl_sync(0xFFFFFFFFu, levels_done, b);
+                    if (action == 1u) {
+                        ++i;
+                        const uint32_t nkb = __shfl_sync(0xFFFFFFFFu, (w[1].y - w[1].x + kBlockK - 1) / kBlockK, b);   // TileDesc::k1, k0
+                        next_batch = nkb <= 4u ? 4u : 1u;
+                    }
+                    if (action >= 2u) stop = true;
+                }
+                batch = next_batch;
             }
         }
     } else if (warp == kTmaWarp) {
