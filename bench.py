@@ -250,6 +250,35 @@ def plan_summary(plan, n_gemms, n_devices):
             "modelled_step_makespan_ms": plan.step_makespan_ns / 1e6}
 
 
+def library_gemm_here(torch, dev, local, warm_s=1.5, timed_s=1.0, n=8192):
+    """The vendor library's bf16 GEMM (n^3) on THIS GPU, the way the pool's sustained figure was taken: back to back
+    until the power cap has pulled the clocks down, then timed with CUDA events, SM clock sampled meanwhile.  Context
+    for the roofline fraction (GPUs of one pool differ by several percent under the same cap); not on any timed path."""
+    a = torch.randn(n, n, device=dev).to(torch.bfloat16)
+    b = torch.randn(n, n, device=dev).to(torch.bfloat16)
+    c = torch.empty(n, n, device=dev, dtype=torch.bfloat16)
+    reps, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < warm_s:
+        for _ in range(20):
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize()
+        reps += 20
+    per_s = reps / (time.perf_counter() - t0)
+    k = max(20, int(per_s * timed_s))
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(k):
+        torch.matmul(a, b, out=c)
+    e1.record()
+    torch.cuda.synchronize()
+    clk = sampler.stop()
+    ms = e0.elapsed_time(e1) / k
+    return {"tflops": 2.0 * n ** 3 / (ms * 1e-3) / 1e12, "sm_mhz": clk.get("sm_mhz"), "reasons": clk.get("reasons"),
+            "how": f"torch.matmul bf16 {n}^3, {k} calls back to back after {warm_s} s of the same"}
+
+
 def quick_leg(cl, ci, torch, dev, name, cfg, scale, opts, mode, min_s=0.6, tensors=None, bf16_out=False, consume=True):
     """Plans the workload, runs it for at least `min_s` seconds untimed, then times the same number of
     steps again: step / exec / assembly times from CUDA events on the launching stream."""
@@ -570,6 +599,12 @@ def run_ours(args):
                 others.append({"name": name, "error": repr(e)})
             torch.cuda.empty_cache()
 
+    lib_here = None
+    if rank == 0 and not args.no_library_gemm:
+        try:
+            lib_here = library_gemm_here(torch, dev, local)
+        except Exception as e:                              # context only: never costs the line
+            lib_here = {"error": repr(e)}
     peaks, peak_kind = load_peaks()
     exec_tflops = flops / (exec_ms * 1e-3) / 1e12
     sm_mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None
@@ -629,7 +664,9 @@ def run_ours(args):
                                   f"{step_s:.1f} s of back-to-back steps (power-capped steady state)",
                      "frac_of_burst": exec_tflops / peaks["bf16_tflops"], "frac_of_nominal": exec_tflops / NOMINAL_BF16_TFLOPS,
                      "flop_per_clk_per_sm": flop_per_clk_per_sm,
-                     "frac_of_tensor_peak_per_clk": flop_per_clk_per_sm / 8192.0 if flop_per_clk_per_sm else None},
+                     "frac_of_tensor_peak_per_clk": flop_per_clk_per_sm / 8192.0 if flop_per_clk_per_sm else None,
+                     "library_gemm_this_gpu": (dict(lib_here, frac=exec_tflops / lib_here["tflops"])
+                                               if lib_here and "tflops" in lib_here else lib_here)},
         "roofline_assemble": roofline_assemble,
         "e2e": {"value": e2e_value if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": plan.num_launches * args.steps,
@@ -664,6 +701,7 @@ def main():
     ap.add_argument("--bf16-out", action="store_true", help="C in bf16 (rounded from the fp32 sums) instead of fp32")
     ap.add_argument("--min-warm-s", type=float, default=1.5, help="warm up for at least this long before the timed steps")
     ap.add_argument("--no-other", action="store_true", help="skip the short legs on other modes and workloads")
+    ap.add_argument("--no-library-gemm", action="store_true", help="skip the vendor library's GEMM on this GPU (context for the roofline)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
