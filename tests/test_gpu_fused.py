@@ -253,3 +253,41 @@ def test_row_granule_256_plan():
     run.exec_fused(); run.assemble(); p.check_status()
     for g, got, want in zip(w.gemms, run.results(), ref):
         assert np.array_equal(got.astype(np.float64), want), g.name
+
+
+def test_short_pairs_straight_to_c_with_dropped_tasks():
+    """Pairs of one to four K-blocks (attention-shaped GEMMs: the scheduler takes their tickets four at
+    a time) whose blocks go straight to C as bulk stores: exact against the oracle on integer inputs.
+    With one task of every second GEMM dropped, pairs that have nothing to run are skipped inside a batch of
+    tickets, the bookkeeping names exactly the missing tasks, and the reissue completes C to the same bits."""
+    w = ci.config(6, 4)                                  # 64 heads: K = 64 (scores) and K = 256 (context)
+    ts = ci.make_tensors(w, integer=True)
+    p, op = lib_plan_for(w), oracle_plan_for(w)
+    A, B = oracle_operands(w, ts)
+    ref = nm.assemble(op, nm.execute(op, A, B))
+    run = GpuRun(w, ts, p)
+    run.exec_opts(direct=True, finish=True); run.assemble(); p.check_status()
+    good = run.results()
+    for gi, g in enumerate(w.gemms):
+        assert np.array_equal(good[gi].astype(np.float64), ref[gi]), g.name
+    done = p.done_counts()
+    assert all(done[i] == p.task_num_tiles(i) for i in range(p.num_tasks))
+
+    p2 = lib_plan_for(w)
+    t = p2.tasks()
+    # the first task of every second GEMM that runs on at least two devices (its owner is lost for that GEMM;
+    # the others survive and take the replacement pieces)
+    failed = np.array([int(t[t["gemm"] == gi]["id"][0]) for gi in range(0, len(w.gemms), 2)
+                       if len(set(t[t["gemm"] == gi]["dev"].tolist())) >= 2], dtype=np.uint32)
+    assert len(failed) >= len(w.gemms) // 4
+    p2.set_drops(failed)
+    run2 = GpuRun(w, ts, p2)
+    run2.exec_opts(direct=True, finish=True); run2.assemble()
+    assert p2.status() == -9
+    lost = set(failed.tolist())
+    done = p2.done_counts()
+    assert all((done[i] == 0) == (i in lost) for i in range(p2.num_tasks))
+    run2.reissue(failed); run2.assemble()
+    assert p2.status() == 0
+    for g, a, b in zip(w.gemms, good, run2.results()):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), g.name
