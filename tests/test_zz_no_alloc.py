@@ -3,6 +3,8 @@
 cudaMalloc): its tables live in a fixed array inside the library instead of buffers allocated on
 first use.  It must give exactly what cleave_assemble gives, call after call, although every call
 reuses the same array.  Collected last on purpose: a failure here cannot hide the other tests."""
+import gc
+
 import numpy as np
 import pytest
 
@@ -60,11 +62,18 @@ def test_no_device_memory_is_taken_by_the_call():
     fresh = lib_plan_for(w, kslice_max=512)                 # same plan, host tables only: no device state yet
     out = [torch.full_like(c, float("nan")) for c in run.C]
     torch.cuda.synchronize()
-    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
-    fresh.assemble_static(run.partials, out)
-    torch.cuda.synchronize()
-    assert torch.cuda.mem_get_info()[0] == free0
-    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    # (tensors of earlier tests that only the garbage collector can free are freed now, and the collector rests
+    # during the call: the figures below must not move for reasons that are not the call's)
+    gc.collect()
+    gc.disable()
+    try:
+        free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        fresh.assemble_static(run.partials, out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0
+        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    finally:
+        gc.enable()
     for g, a, b in zip(w.gemms, ref, out):
         assert np.array_equal(a.view(np.uint32), b.cpu().numpy().view(np.uint32)), g.name
     # two calls back to back on one stream, nothing in between: the second call's tables wait for the first's kernels
