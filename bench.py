@@ -588,6 +588,9 @@ def run_ours(args):
                 ("same workload, bf16 outputs", args.config, args.scale, base, "fused", True, shared)]
         if args.gran_m is None:
             legs.append(("same workload, row granule 256", args.config, args.scale, dict(base, gran_m=256), "fused", False, shared))
+        if args.kslice_max is None:                        # the K-slice cap's sweep: half the default, and no cap (one slice per GEMM)
+            legs.append(("same workload, K-slices of at most 2048", args.config, args.scale, dict(base, kslice_max=2048), "fused", False, shared))
+            legs.append(("same workload, no K-slice cap (every GEMM one slice)", args.config, args.scale, dict(base, kslice_max=0), "fused", False, shared))
         if args.config == 3 and args.scale == 1:
             legs += [("GPT-2-small-shaped layer, 64 devices", 2, 1, {}, "fused", False, {}),
                      ("Llama-13B-shaped layer, 4096 devices", 5, 1, {}, "fused", False, {}),
