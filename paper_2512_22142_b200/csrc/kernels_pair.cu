@@ -33,6 +33,11 @@
 // block; under MODE_CONSUME it does not even store that block: it is used up on arrival).  A strip that
 // only turns out to be last after storing its block reads all blocks back.
 // Under MODE_BF16 values written to C are rounded to bf16.
+// A whole 32 x 32 chunk that goes straight to an fp32 C leaves as one bulk tensor store from the warp's
+// staging tile (the warp issues it and moves on); everything else is written with float4 row stores.
+// The bookkeeping counts of a strip (its tasks' done words, its level's counter) must follow a fence
+// that waits for the strip's stores; a warp owes them and pays several strips with one fence when it
+// would wait anyway.
 //
 // DAG levels: tiles are ordered by level, and before the scheduler hands out the first tile of a
 // level it waits until every strip of the lower levels has been written (a counter per level that
