@@ -594,7 +594,8 @@ def run_ours(args):
         if args.config == 3 and args.scale == 1:
             legs += [("GPT-2-small-shaped layer, 64 devices", 2, 1, {}, "fused", False, {}),
                      ("Llama-13B-shaped layer, 4096 devices", 5, 1, {}, "fused", False, {}),
-                     ("attention GEMMs of 1024 heads as tasks, 64 devices", 6, 1, {}, "fused", False, {})]
+                     ("attention GEMMs of 1024 heads as tasks, 64 devices", 6, 1, {}, "fused", False, {}),
+                     ("attention GEMMs of 1024 heads as tasks, bf16 outputs", 6, 1, {}, "fused", True, {})]
         for name, cfg, scale, o, mode, b16, kw in legs:
             try:
                 others.append(quick_leg(cl, ci, torch, dev, name, cfg, scale, o, mode, bf16_out=b16, **kw))

@@ -25,7 +25,7 @@ struct DeviceState {
     uint32_t* failed_ids = nullptr;
     unsigned int* words = nullptr;    // [0] ticket, [1] status, [2] failed count
     CUtensorMap* maps = nullptr;
-    CUtensorMap* c_maps = nullptr;    // per GEMM: C as an fp32 matrix, 32 x 32 boxes (the exec kernel's bulk stores)
+    CUtensorMap* c_maps = nullptr;    // per GEMM two maps of C, 32 x 32 boxes (the exec kernel's bulk stores): as fp32, as bf16
     AsmItem* asm_items = nullptr;
     AsmRef* asm_refs = nullptr;
     void** c_ptrs = nullptr;
@@ -96,17 +96,19 @@ int encode_map_groups(CUtensorMap* out, const void* base, uint64_t rows, uint64_
     return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
 }
 
-// fp32 tensor map over a row-major [rows x cols] matrix C: boxes of 32 x 32 elements (128-byte rows,
-// 128-byte swizzle): what an epilogue warp of the exec kernel stores with one bulk operation.
-int encode_c_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols) {
+// Tensor map over a row-major [rows x cols] matrix C, fp32 or bf16: boxes of 32 x 32 elements (rows of 128
+// bytes with the 128-byte swizzle, resp. 64 bytes with the 64-byte swizzle): what an epilogue warp of the exec
+// kernel stores with one bulk operation.
+int encode_c_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, bool bf16) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return CLEAVE_E_CUDA;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 4};
+    cuuint64_t strides[1] = {cols * (bf16 ? 2u : 4u)};
     cuuint32_t box[2] = {32, 32};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+    CUresult r = fn(out, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
+                    dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : CLEAVE_E_CUDA;
 }
@@ -135,7 +137,7 @@ int create_device_state(cleave_plan_s* p, cudaStream_t st, DeviceState* d) {
     RC_TRY(dev_alloc(&d->words, 4));
     CU_TRY(cudaMemsetAsync(d->words, 0, 4 * sizeof(unsigned int), st));
     RC_TRY(dev_alloc(&d->maps, kMapsPerGemm * ng));
-    RC_TRY(dev_alloc(&d->c_maps, ng));
+    RC_TRY(dev_alloc(&d->c_maps, 2 * ng));
     RC_TRY(dev_alloc(&d->c_ptrs, ng));
     RC_TRY(dev_alloc(&d->ldcs, ng));
     std::vector<uint32_t> ldc;
@@ -255,14 +257,17 @@ int upload_c_ptrs(cleave_plan_s* p, void* const* C, cudaStream_t st) {
     if (d->last_c.size() != n || !std::equal(C, C + n, d->last_c.begin())) {
         d->last_c.assign(C, C + n);
         CU_TRY(cudaMemcpyAsync(d->c_ptrs, d->last_c.data(), n * sizeof(void*), cudaMemcpyHostToDevice, st));
-        // fp32 views of the outputs for bulk stores (the kernel uses one only for fp32 output with N % 4 == 0)
-        std::vector<CUtensorMap> host(n);
+        // views of the outputs for bulk stores: as fp32 (used when C holds fp32 and N % 4 == 0) and as bf16 (when C
+        // holds bf16 and N % 8 == 0); the buffer is whichever the caller made it, the other view is never used
+        std::vector<CUtensorMap> host(2 * n);
         for (size_t i = 0; i < n; ++i) {
             const cleave_gemm_t& g = p->gemms[i];
-            if (g.N % 4 == 0) RC_TRY(encode_c_map(&host[i], C[i], g.M, g.N));
-            else std::memset(&host[i], 0, sizeof(CUtensorMap));
+            if (g.N % 4 == 0) RC_TRY(encode_c_map(&host[2 * i], C[i], g.M, g.N, false));
+            else std::memset(&host[2 * i], 0, sizeof(CUtensorMap));
+            if (g.N % 8 == 0) RC_TRY(encode_c_map(&host[2 * i + 1], C[i], g.M, g.N, true));
+            else std::memset(&host[2 * i + 1], 0, sizeof(CUtensorMap));
         }
-        CU_TRY(cudaMemcpyAsync(d->c_maps, host.data(), n * sizeof(CUtensorMap), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(d->c_maps, host.data(), 2 * n * sizeof(CUtensorMap), cudaMemcpyHostToDevice, st));
     }
     return 0;
 }

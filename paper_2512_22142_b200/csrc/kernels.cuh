@@ -40,7 +40,7 @@ struct ExecParams {
     uint32_t tile_end;              // the ticket runs up to here
     unsigned int* ticket;
     const CUtensorMap* maps;        // kMapsPerGemm per GEMM
-    const CUtensorMap* c_maps;      // per GEMM: C as fp32 with 32 x 32 boxes (bulk stores of blocks that go straight to C)
+    const CUtensorMap* c_maps;      // per GEMM: C with 32 x 32 boxes as fp32, then as bf16 (bulk stores of blocks that go straight to C)
     float* partials;                // arena
     void* const* c_ptrs;            // per GEMM: C (fp32, or bf16 under MODE_BF16)
     uint32_t* done;                 // per task: finished half-tiles x epilogue warps

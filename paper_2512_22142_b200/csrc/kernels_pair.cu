@@ -200,6 +200,18 @@ __device__ __forceinline__ void stage_row(float* stage_tile, uint32_t row, const
     for (uint32_t j = 0; j < 8; ++j)
         base[j ^ (row & 7u)] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
 }
+// The same chunk rounded to bf16: 32 rows of 64 bytes, the four 16-byte chunks of row r stored at chunk position
+// j ^ ((r >> 1) & 3) (the 64-byte swizzle pattern of the bf16 tensor map of C; a warp's 512 bytes per step
+// touch every bank four times, the minimum).
+__device__ __forceinline__ void stage_row_bf16(float* stage_tile, uint32_t row, const uint32_t (&v)[32]) {
+    uint4* base = reinterpret_cast<uint4*>(stage_tile) + row * 4u;
+#pragma unroll
+    for (uint32_t j = 0; j < 4; ++j)
+        base[j ^ ((row >> 1) & 3u)] = make_uint4(pack_bf16(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1])),
+                                                 pack_bf16(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3])),
+                                                 pack_bf16(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5])),
+                                                 pack_bf16(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7])));
+}
 __device__ __forceinline__ float4 staged_f4(const float* stage_tile, uint32_t row, uint32_t col4) {      // columns 4*col4 .. +3
     return reinterpret_cast<const float4*>(stage_tile)[row * 8u + (col4 ^ (row & 7u))];
 }
@@ -632,9 +644,10 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
             // a block of a one-slice GEMM is final: it may go straight to its place in C
             const bool direct = (P.mode & MODE_DIRECT) && (flags & TILE_SINGLE);
             const bool to_bf16 = direct && out_bf16;
-            const bool bulk_ok = direct && !out_bf16 && rows_here == 32u && ((ldc | n_col) & 3u) == 0u;
+            const bool bulk_ok = direct && rows_here == 32u && ((ldc | n_col) & (out_bf16 ? 7u : 3u)) == 0u;
+            const CUtensorMap* c_map = P.c_maps + 2u * gemm + (out_bf16 ? 1u : 0u);
             if (bulk_ok && gemm != c_map_gemm) {
-                if (lane == 0) tensormap_acquire(P.c_maps + gemm);
+                if (lane == 0) tensormap_acquire(c_map);
                 c_map_gemm = gemm;
             }
             const uint64_t c_off = (uint64_t)h_m_row * ldc + n_col;            // the half-tile's (0, 0) in C
@@ -708,17 +721,18 @@ exec_pair_kernel(const __grid_constant__ ExecParams P) {
                 }
                 if (!live_chunk) continue;
                 staging_free();
-                stage_row(stage_tile, lane, v);
                 if (bulk_ok && ct + 32u <= cols) {
+                    if (to_bf16) stage_row_bf16(stage_tile, lane, v); else stage_row(stage_tile, lane, v);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the staged values, before the bulk store reads them
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d(P.c_maps + gemm, smem_u32(stage_tile), (int32_t)(n_col + ct), (int32_t)(h_m_row + row0));
+                        tma_store_2d(c_map, smem_u32(stage_tile), (int32_t)(n_col + ct), (int32_t)(h_m_row + row0));
                         bulk_commit();
                     }
                     bulk_reading = bulk_flying = true;
                     continue;
                 }
+                stage_row(stage_tile, lane, v);
                 __syncwarp();
                 const uint32_t ld = direct ? ldc : sg_ld;
                 const uint64_t out_off = direct ? c_off + (uint64_t)row0 * ldc + ct : sg_out_off + (uint64_t)row0 * sg_ld + c0;
