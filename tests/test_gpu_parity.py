@@ -36,6 +36,14 @@ def _run_and_compare_exact(w, opts=None, integer=True):
             assert_within_tolerance(out[gi], ref[gi], nm.abs_bound(A[gi], B[gi]), what=g.name)
     done = p.done_counts()
     assert all(done[i] == p.task_num_tiles(i) for i in range(p.num_tasks))
+    # the fused write-out (blocks of one-slice GEMMs straight to C, bulk stores where a chunk is whole and aligned,
+    # K-split cells summed in the kernel) must give the same bits on the same plan
+    fused = GpuRun(w, ts, p)
+    fused.exec_opts(direct=True, finish=True)
+    fused.assemble()
+    p.check_status()
+    for gi, g in enumerate(w.gemms):
+        assert np.array_equal(out[gi].view(np.uint32), fused.results()[gi].view(np.uint32)), f"{g.name}: fused write-out differs"
     return p, op, run, ref
 
 
